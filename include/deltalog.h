@@ -1,0 +1,157 @@
+/*
+ * deltalog.h -- C ABI of the DeltaLog recurrent-state decode library (sm_100a).
+ *
+ * The library keeps the recurrent state of a linear-attention layer as a dense fp32 base plus a
+ * bounded log of compact per-token factors (Section 3.1 of the paper):
+ *
+ *     S_t = D(lbar) S_base + sum_{i < len} D(lbar - Lambda[i]) K[i] U[i]^T          (Eq. 6)
+ *
+ * with D(l) = diag(exp(l)) acting on the key dimension (rows), lbar the log-decay accumulated
+ * since the last materialisation and Lambda[i] its snapshot when entry i was appended.  Because
+ * Lambda[len-1] is lbar by construction (Eq. 4 stores lbar after it absorbed the token's decay),
+ * lbar is not stored separately: lbar = Lambda[len-1], or 0 for an empty log.
+ *
+ * Operators (Table 1; the gate is passed in log space, lambda_t = log alpha_t or log w_t):
+ *   DELTALOG_GDN    scalar decay per head, delta rule:   b_t = beta_t (v_t - (D(lambda_t) S_{t-1})^T k_t)
+ *   DELTALOG_KDA    per-key decay,          delta rule:   same b_t
+ *   DELTALOG_RWKV6  per-key decay, b_t = v_t, output read from S_{t-1} plus the bonus term
+ * All use a_t = k_t and S_t = D(lambda_t) S_{t-1} + a_t b_t^T (Eq. 3).
+ *
+ * General rules for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller; descriptor structs are HOST
+ *     memory, read during the call only.  The library allocates nothing and keeps no state.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and never synchronise.
+ *   - Tensors are dense, row-major in the index order written beside them, 16-byte aligned.
+ *   - Return value: DELTALOG_OK (0) when the work was launched; any other code means the
+ *     arguments were rejected on the host and nothing was launched.
+ *   - Conditions only visible on the device (a row whose log is already full, a slot index out of
+ *     range) make the kernel skip that row, OR a bit into *state->status (if non-NULL) and carry
+ *     on; kernels never trap.  Rows with slot index < 0 are padding and are skipped silently.
+ *   - The same slot must not appear twice in one call.
+ *   - Supported shapes: d_k == d_v in {64, 128}; 1 <= cap <= 64; klog_dtype == io_dtype;
+ *     ulog_dtype == F32 for GDN / KDA and == io_dtype for RWKV6.
+ */
+#ifndef DELTALOG_H
+#define DELTALOG_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { DELTALOG_GDN = 0, DELTALOG_KDA = 1, DELTALOG_RWKV6 = 2 } deltalog_op;
+typedef enum { DELTALOG_F32 = 0, DELTALOG_BF16 = 1 } deltalog_dtype;
+
+/* host-side return codes */
+enum {
+    DELTALOG_OK = 0,
+    DELTALOG_ERR_INVALID_ARG = 1,       /* NULL where a pointer is required, B < 0, bad enum, misaligned pointer */
+    DELTALOG_ERR_UNSUPPORTED_SHAPE = 2, /* d_k / d_v / dtype combination outside the supported set */
+    DELTALOG_ERR_CAP_RANGE = 3,         /* cap outside 1..64 */
+    DELTALOG_ERR_CUDA = 4               /* the CUDA runtime refused the launch or a copy */
+};
+
+/* bits OR-ed into *status by kernels */
+enum {
+    DELTALOG_STATUS_LOG_FULL = 1, /* decode on a (slot, head) whose log already holds cap entries: row skipped */
+    DELTALOG_STATUS_BAD_SLOT = 2, /* slot index >= num_slots: row skipped */
+    DELTALOG_STATUS_TIMEOUT = 4   /* a bounded wait inside a kernel gave up: results of that launch are invalid */
+};
+
+/* Problem description (host memory). */
+typedef struct {
+    int32_t op;         /* deltalog_op */
+    int32_t num_slots;  /* size of the state pool */
+    int32_t H;          /* heads */
+    int32_t d_k, d_v;   /* head dimensions */
+    int32_t cap;        /* log capacity: appends possible between two merges */
+    int32_t io_dtype;   /* deltalog_dtype of q, k, v, out */
+    int32_t klog_dtype; /* deltalog_dtype of K_log */
+    int32_t ulog_dtype; /* deltalog_dtype of U_log */
+    float scale;        /* multiplies the output of GDN / KDA (ignored for RWKV6) */
+} deltalog_desc;
+
+/* Physical state (Section 3.1).  Device pointers, caller-owned. d_lambda = 1 (GDN) or d_k. */
+typedef struct {
+    float *S_base;     /* [num_slots, H, d_k, d_v] fp32 dense base                                  */
+    void *K_log;       /* [num_slots, H, cap, d_k] key-side factors a_t                             */
+    void *U_log;       /* [num_slots, H, cap, d_v] value-side factors b_t                           */
+    float *decay_log;  /* [num_slots, H, cap, d_lambda] Lambda: cumulative log-decay snapshots, fp32 */
+    int32_t *log_len;  /* [num_slots, H] live entries, 0..cap; zero it for a fresh or reused slot   */
+    int32_t *status;   /* one word of DELTALOG_STATUS_* bits, or NULL                               */
+} deltalog_state;
+
+/*
+ * One decode token for B rows (Algorithm 1, append branch; Eq. 4).
+ * Row b updates slot slot_idx[b] (slot b if slot_idx is NULL), all H heads.
+ * Reads S_base once and the live log entries; computes `out`; appends (k_t, b_t, lbar + lambda_t)
+ * as entry log_len and increments log_len.  Never writes S_base.
+ *
+ *   q, k, v  [B, H, d]  io_dtype (q is the receptance r for RWKV6)
+ *   g        log-decay lambda_t <= 0, fp32: [B, H] for GDN, [B, H, d_k] for KDA / RWKV6
+ *   beta     [B, H] fp32 for GDN / KDA; ignored (may be NULL) for RWKV6
+ *   u_bonus  [H, d_k] fp32 for RWKV6; ignored (may be NULL) otherwise
+ *   out      [B, H, d_v] io_dtype;  GDN / KDA: scale * S_t^T q_t;
+ *            RWKV6: S_{t-1}^T r_t + (r_t . (u_bonus (.) k_t)) v_t
+ */
+int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state, const void *q,
+                         const void *k, const void *v, const float *g, const float *beta,
+                         const float *u_bonus, const int32_t *slot_idx, int32_t B, void *out,
+                         void *stream);
+
+/*
+ * Materialise the log into the base (Eq. 5 without the current-token term):
+ *     S_base <- D(lbar) S_base + sum_i D(lbar - Lambda[i]) K[i] U[i]^T ;  log_len <- 0
+ * for the n slots listed in slot_idx (slots 0..n-1 if NULL), all heads.  A (slot, head) with an
+ * empty log is left untouched (no dense write).  With only_if_full != 0, (slot, head) pairs whose
+ * log holds fewer than cap entries are skipped as well, so one call over the whole batch serves
+ * sequences whose merge boundaries are staggered.
+ */
+int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const int32_t *slot_idx,
+                   int32_t n, int32_t only_if_full, void *stream);
+
+/*
+ * The eager dense comparator (Section 2.3): the same token update applied directly to a dense
+ * state S [num_slots, H, d_k, d_v] fp32, which is read and rewritten in full on every call.
+ * Token arguments and `out` as for deltalog_decode_step; `status` (may be NULL) receives
+ * DELTALOG_STATUS_BAD_SLOT bits.
+ */
+int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, const void *k,
+                        const void *v, const float *g, const float *beta, const float *u_bonus,
+                        const int32_t *slot_idx, int32_t B, void *out, int32_t *status, void *stream);
+
+/*
+ * deltalog_decode_step for callers whose token tensors live in HOST memory (pinned for the copies
+ * to be asynchronous): copies q, k, v, g, beta (and nothing else) to the caller-provided device
+ * staging buffers on `stream`, runs the decode step there and copies `out` back to host_out.
+ * The state, u_bonus and slot_idx stay device-resident.  Staging buffers have the shapes of the
+ * tensors they stage.  Returns after enqueuing; synchronise the stream before reading host_out.
+ */
+typedef struct {
+    void *q, *k, *v; /* device, [B, H, d] io_dtype */
+    float *g;        /* device, shape of g */
+    float *beta;     /* device, [B, H]; unused for RWKV6 */
+    void *out;       /* device, [B, H, d_v] io_dtype */
+} deltalog_staging;
+
+int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *state,
+                              const deltalog_staging *staging, const void *host_q,
+                              const void *host_k, const void *host_v, const float *host_g,
+                              const float *host_beta, const float *u_bonus,
+                              const int32_t *slot_idx, int32_t B, void *host_out, void *stream);
+
+/* Human-readable text for a host return code (static storage). */
+const char *deltalog_status_string(int code);
+
+/* Library version, major * 10000 + minor * 100 + patch. */
+int deltalog_version(void);
+
+/* Number of kernels the library has launched in this process (host counter, all entry points). */
+uint64_t deltalog_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DELTALOG_H */

@@ -1,0 +1,113 @@
+"""TEST INFRASTRUCTURE -- the base-plus-log schedule in fp64 numpy. Not part of the product path.
+
+The physical state of the deferred representation (Section 3.1): a dense base ``S_base``, a
+cumulative log-decay ``lbar`` since the last materialisation, a bounded log of compact factors
+``K_log[i] = a``, ``U_log[i] = b``, one log-decay snapshot ``Lam_log[i]`` per entry, and the live
+length ``length``.  The functions below follow Algorithm 1 with the cycle split the way this
+library splits it: the decode step always appends (Eq. 4), and materialisation (Eq. 5 without the
+current-token term) is a separate, token-less merge.
+
+Everything is written for clarity, not speed: every readout first materialises the logical state
+with Eq. 6 as a dense matrix and then applies the operator's definition to it.  Python loops run
+over units; use small N, T.
+
+Pins (tests/test_oracle_pins.py): after every append and every merge the state materialised by
+Eq. 6 equals the eager recurrence of ``eager_oracle.c`` to ~1e-13, for every capacity, which is
+the closure property the paper proves below Eq. 6; the eager recurrence itself is pinned against
+closed forms there.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+GDN, KDA, RWKV6 = 0, 1, 2
+
+
+class LogState:
+    """Base + bounded log for ``N`` independent (sequence, head) units (Section 3.1)."""
+
+    def __init__(self, op: int, S0: np.ndarray, cap: int):
+        S0 = np.asarray(S0, dtype=np.float64)
+        self.op = int(op)
+        self.N, self.d_k, self.d_v = S0.shape
+        self.cap = int(cap)
+        self.d_lambda = 1 if self.op == GDN else self.d_k
+        self.S_base = S0.copy()
+        self.lbar = np.zeros((self.N, self.d_lambda))
+        self.K_log = np.zeros((self.N, self.cap, self.d_k))
+        self.U_log = np.zeros((self.N, self.cap, self.d_v))
+        self.Lam_log = np.zeros((self.N, self.cap, self.d_lambda))
+        self.length = np.zeros(self.N, dtype=np.int64)
+
+
+def _row_scale(ell: np.ndarray, d_k: int) -> np.ndarray:
+    """exp(ell) as a length-d_k vector (a scalar decay is shared by all key coordinates)."""
+    ell = np.asarray(ell, dtype=np.float64).reshape(-1)
+    return np.exp(np.broadcast_to(ell, (d_k,)) if ell.size == 1 else ell)
+
+
+def materialize_unit(S_base, lbar, K_log, U_log, Lam_log, length) -> np.ndarray:
+    """Eq. 6 for one unit: S = D(lbar) S_base + sum_{i<length} D(lbar - Lam[i]) K[i] U[i]^T."""
+    d_k = S_base.shape[0]
+    S = _row_scale(lbar, d_k)[:, None] * S_base
+    for i in range(int(length)):
+        w = _row_scale(np.asarray(lbar) - np.asarray(Lam_log[i]), d_k)
+        S = S + np.outer(w * K_log[i], U_log[i])
+    return S
+
+
+def materialize(st: LogState) -> np.ndarray:
+    """Eq. 6 for every unit -> [N, d_k, d_v]."""
+    return np.stack([
+        materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], st.length[n])
+        for n in range(st.N)
+    ])
+
+
+def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float = 1.0) -> np.ndarray:
+    """One token through Algorithm 1's append branch for every unit; returns ``out [N, d_v]``.
+
+    ``q,k [N,d_k]``, ``v [N,d_v]``, ``lam [N,d_lambda]``, ``beta [N]`` (GDN/KDA), ``bonus [N,d_k]`` (RWKV6).
+    Raises if a unit's log is already full (the caller merges first).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    lam = np.asarray(lam, dtype=np.float64).reshape(st.N, st.d_lambda)
+    out = np.empty((st.N, st.d_v))
+    for n in range(st.N):
+        L = int(st.length[n])
+        if L >= st.cap:
+            raise RuntimeError(f"unit {n}: log full (length {L} == capacity); merge first")
+        # line 1: readouts defined on the pre-update logical state
+        S_prev = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L)
+        # line 2: fold the token's log-decay into the cumulative log-decay
+        st.lbar[n] = st.lbar[n] + lam[n]
+        S_decayed = _row_scale(lam[n], st.d_k)[:, None] * S_prev
+        # line 3: update factors (a, b) and the output of the original recurrence
+        a = k[n]
+        if st.op == RWKV6:
+            b = v[n]
+            out[n] = S_prev.T @ q[n] + float(np.sum(q[n] * bonus[n] * k[n])) * v[n]
+        else:
+            b = float(beta[n]) * (v[n] - S_decayed.T @ k[n])
+        # lines 4-5 / Eq. 4: append (a, b, lbar) into slot L; the base is untouched
+        st.K_log[n, L] = a
+        st.U_log[n, L] = b
+        st.Lam_log[n, L] = st.lbar[n]
+        st.length[n] = L + 1
+        if st.op != RWKV6:
+            S_new = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L + 1)
+            out[n] = scale * (S_new.T @ q[n])
+    return out
+
+
+def merge(st: LogState, only_if_full: bool = False) -> None:
+    """Eq. 5 without the current-token term: fold the log into the base, reset lbar and length."""
+    for n in range(st.N):
+        L = int(st.length[n])
+        if L == 0 or (only_if_full and L < st.cap):
+            continue
+        st.S_base[n] = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L)
+        st.lbar[n] = 0.0
+        st.length[n] = 0

@@ -1,0 +1,274 @@
+"""Pins for the CPU oracle: closed forms, invariants and special cases fixed by the paper and by
+linear algebra.  None of the expected values below is produced by the oracle's own arithmetic.
+
+What each pin would catch:
+  * explicit product of (I - beta k k^T) D(lambda) factors  -> wrong order of decay / correction /
+    update, decay applied to columns instead of rows, wrong sign in the correction;
+  * unrolled sum of outer products for RWKV6                -> decay applied to the new token,
+    readout taken after instead of before the update, bonus on the wrong operand;
+  * identity / pure-decay invariants, delta-rule recall     -> dropped terms, beta misplaced;
+  * KDA with equal channels == GDN, superposition           -> per-key indexing, hidden non-linearity;
+  * Eq. 1 prefix sums                                       -> transposed state (k v^T vs v k^T).
+"""
+import numpy as np
+import pytest
+
+import oracle
+from oracle import GDN, KDA, RWKV6, logical
+
+RNG = np.random.default_rng(12345)
+
+
+def rand_inputs(op, T, N, dk, dv, rng=None, unit_keys=False):
+    rng = rng or np.random.default_rng(T * 1000 + N * 100 + dk * 10 + dv + op)
+    dl = 1 if op == GDN else dk
+    S0 = rng.normal(0, 0.3, (N, dk, dv))
+    q = rng.normal(0, 1, (T, N, dk))
+    k = rng.normal(0, 1, (T, N, dk))
+    if unit_keys:
+        k /= np.linalg.norm(k, axis=-1, keepdims=True)
+    v = rng.normal(0, 1, (T, N, dv))
+    lam = -np.log1p(np.exp(rng.normal(0, 1, (T, N, dl))))
+    beta = 1 / (1 + np.exp(-rng.normal(0, 1, (T, N))))
+    bonus = rng.normal(0, 0.5, (N, dk))
+    return S0, q, k, v, lam, beta, bonus
+
+
+def roll(op, S0, q, k, v, lam, beta, bonus, **kw):
+    if op == RWKV6:
+        return oracle.eager_rollout(op, S0, q, k, v, lam, bonus=bonus, **kw)
+    return oracle.eager_rollout(op, S0, q, k, v, lam, beta=beta, **kw)
+
+
+# ---------------------------------------------------------------------------------------------
+# GDN / KDA: explicit dense transition matrices A_s = (I - beta_s k_s k_s^T) D(lambda_s)
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("op", [GDN, KDA])
+@pytest.mark.parametrize("T,dk,dv", [(1, 2, 3), (5, 4, 3), (8, 8, 5), (7, 3, 8)])
+def test_delta_rule_matches_explicit_product_of_factors(op, T, dk, dv):
+    N = 3
+    S0, q, k, v, lam, beta, _ = rand_inputs(op, T, N, dk, dv)
+    scale = 0.7
+    res = oracle.eager_rollout(op, S0, q, k, v, lam, beta=beta, scale=scale,
+                               snapshot_at=range(1, T + 1))
+    for n in range(N):
+        A = []
+        for s in range(T):
+            dvec = np.exp(np.broadcast_to(lam[s, n], (dk,)))
+            A.append((np.eye(dk) - beta[s, n] * np.outer(k[s, n], k[s, n])) @ np.diag(dvec))
+        for t in range(1, T + 1):
+            P = np.eye(dk)
+            for s in range(t):
+                P = A[s] @ P
+            S_t = P @ S0[n]
+            for s in range(t):
+                Q = np.eye(dk)
+                for r in range(s + 1, t):
+                    Q = A[r] @ Q
+                S_t = S_t + Q @ (beta[s, n] * np.outer(k[s, n], v[s, n]))
+            np.testing.assert_allclose(res["snapshots"][t - 1, n], S_t, rtol=0, atol=1e-12)
+            np.testing.assert_allclose(res["out"][t - 1, n], scale * (S_t.T @ q[t - 1, n]),
+                                       rtol=0, atol=1e-12)
+        np.testing.assert_allclose(res["S"][n], res["snapshots"][T - 1, n], rtol=0, atol=0)
+
+
+@pytest.mark.parametrize("op", [GDN, KDA])
+def test_value_side_factor_is_beta_times_residual_on_decayed_state(op):
+    T, N, dk, dv = 4, 2, 5, 6
+    S0, q, k, v, lam, beta, _ = rand_inputs(op, T, N, dk, dv)
+    res = oracle.eager_rollout(op, S0, q, k, v, lam, beta=beta, snapshot_at=range(1, T + 1))
+    for n in range(N):
+        prev = S0[n]
+        for t in range(T):
+            decayed = np.exp(np.broadcast_to(lam[t, n], (dk,)))[:, None] * prev
+            b = beta[t, n] * (v[t, n] - decayed.T @ k[t, n])
+            np.testing.assert_allclose(res["b"][t, n], b, atol=1e-13)
+            prev = res["snapshots"][t, n]
+
+
+# ---------------------------------------------------------------------------------------------
+# RWKV6: unrolled sum of outer products, bonus readout, Eq. 1 special case
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T,dk,dv", [(1, 2, 2), (6, 4, 3), (8, 8, 4), (5, 2, 8)])
+def test_rwkv6_matches_unrolled_sum_of_outer_products(T, dk, dv):
+    N = 3
+    S0, r, k, v, lam, _, bonus = rand_inputs(RWKV6, T, N, dk, dv)
+    res = oracle.eager_rollout(RWKV6, S0, r, k, v, lam, bonus=bonus, snapshot_at=range(1, T + 1))
+    w = np.exp(lam)
+
+    def closed(n, t):  # S_t, t tokens consumed
+        S = np.prod(w[:t, n], axis=0)[:, None] * S0[n] if t else S0[n].copy()
+        for s in range(t):
+            S = S + (np.prod(w[s + 1:t, n], axis=0) * k[s, n])[:, None] * v[s, n][None, :]
+        return S
+
+    for n in range(N):
+        for t in range(1, T + 1):
+            np.testing.assert_allclose(res["snapshots"][t - 1, n], closed(n, t), atol=1e-12)
+            o = closed(n, t - 1).T @ r[t - 1, n] + np.dot(r[t - 1, n], bonus[n] * k[t - 1, n]) * v[t - 1, n]
+            np.testing.assert_allclose(res["out"][t - 1, n], o, atol=1e-12)
+        np.testing.assert_allclose(res["b"][:, n], v[:, n], atol=0)
+
+
+def test_rwkv6_first_token_from_zero_state_is_pure_bonus():
+    S0, r, k, v, lam, _, bonus = rand_inputs(RWKV6, 1, 2, 4, 3)
+    res = oracle.eager_rollout(RWKV6, np.zeros_like(S0), r, k, v, lam, bonus=bonus)
+    for n in range(2):
+        np.testing.assert_allclose(res["out"][0, n], np.dot(r[0, n], bonus[n] * k[0, n]) * v[0, n], atol=1e-14)
+        np.testing.assert_allclose(res["S"][n], np.outer(k[0, n], v[0, n]), atol=1e-14)
+
+
+def test_rwkv6_without_decay_and_bonus_is_shifted_linear_attention():
+    """w = 1, bonus = 0: S_t is the plain prefix sum of k v^T (Eq. 1) and o_t reads S_{t-1}."""
+    T, N, dk, dv = 6, 2, 3, 4
+    S0, r, k, v, lam, _, bonus = rand_inputs(RWKV6, T, N, dk, dv)
+    res = oracle.eager_rollout(RWKV6, np.zeros_like(S0), r, k, v, np.zeros_like(lam),
+                               bonus=np.zeros_like(bonus), snapshot_at=range(1, T + 1))
+    for n in range(N):
+        prefix = np.cumsum(np.einsum("tj,tc->tjc", k[:, n], v[:, n]), axis=0)
+        np.testing.assert_allclose(res["snapshots"][:, n], prefix, atol=1e-13)
+        np.testing.assert_allclose(res["out"][0, n], 0.0, atol=0)
+        for t in range(1, T):
+            np.testing.assert_allclose(res["out"][t, n], prefix[t - 1].T @ r[t, n], atol=1e-13)
+
+
+# ---------------------------------------------------------------------------------------------
+# invariants and special cases
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("op", [GDN, KDA])
+def test_no_decay_no_write_keeps_state(op):
+    T, N, dk, dv = 5, 2, 4, 4
+    S0, q, k, v, lam, beta, _ = rand_inputs(op, T, N, dk, dv)
+    res = oracle.eager_rollout(op, S0, q, k, v, np.zeros_like(lam), beta=np.zeros_like(beta), scale=2.0)
+    np.testing.assert_allclose(res["S"], S0, atol=0)
+    np.testing.assert_allclose(res["out"], 2.0 * np.einsum("njc,tnj->tnc", S0, q), atol=1e-13)
+    np.testing.assert_allclose(res["b"], 0.0, atol=0)
+
+
+def test_gdn_pure_scalar_decay_is_geometric():
+    T, N, dk, dv = 7, 2, 3, 5
+    S0, q, k, v, lam, beta, _ = rand_inputs(GDN, T, N, dk, dv)
+    c = 0.8
+    res = oracle.eager_rollout(GDN, S0, q, k, v, np.full_like(lam, np.log(c)), beta=np.zeros_like(beta),
+                               snapshot_at=range(1, T + 1))
+    for t in range(1, T + 1):
+        np.testing.assert_allclose(res["snapshots"][t - 1], c ** t * S0, rtol=1e-13)
+
+
+@pytest.mark.parametrize("op", [GDN, KDA])
+def test_delta_rule_recall_with_unit_keys_and_full_write(op):
+    """beta = 1 and ||k|| = 1: the updated state returns exactly v_t for key k_t, whatever the decay."""
+    T, N, dk, dv = 6, 3, 8, 5
+    S0, q, k, v, lam, beta, _ = rand_inputs(op, T, N, dk, dv, unit_keys=True)
+    res = oracle.eager_rollout(op, S0, k.copy(), k, v, lam, beta=np.ones_like(beta))  # query with k itself
+    np.testing.assert_allclose(res["out"], v, atol=1e-12)
+
+
+def test_kda_with_equal_channels_is_gdn():
+    T, N, dk, dv = 6, 2, 5, 4
+    S0, q, k, v, lam, beta, _ = rand_inputs(GDN, T, N, dk, dv)
+    a = oracle.eager_rollout(GDN, S0, q, k, v, lam, beta=beta)
+    b = oracle.eager_rollout(KDA, S0, q, k, v, np.repeat(lam, dk, axis=-1), beta=beta)
+    for key in ("out", "S", "b"):
+        np.testing.assert_allclose(a[key], b[key], rtol=0, atol=1e-14)
+
+
+@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+def test_superposition_in_state_and_values(op):
+    T, N, dk, dv = 5, 2, 4, 3
+    S0, q, k, v, lam, beta, bonus = rand_inputs(op, T, N, dk, dv)
+    rng = np.random.default_rng(7)
+    S0b, vb = rng.normal(size=S0.shape), rng.normal(size=v.shape)
+    r1 = roll(op, S0, q, k, v, lam, beta, bonus)
+    r2 = roll(op, S0b, q, k, vb, lam, beta, bonus)
+    r3 = roll(op, 2 * S0 - 3 * S0b, q, k, 2 * v - 3 * vb, lam, beta, bonus)
+    for key in ("out", "S"):
+        np.testing.assert_allclose(r3[key], 2 * r1[key] - 3 * r2[key], atol=1e-11)
+
+
+@pytest.mark.parametrize("op", [GDN, KDA])
+def test_single_token_from_zero_state(op):
+    S0, q, k, v, lam, beta, _ = rand_inputs(op, 1, 2, 4, 3)
+    res = oracle.eager_rollout(op, np.zeros_like(S0), q, k, v, lam, beta=beta, scale=0.5)
+    for n in range(2):
+        np.testing.assert_allclose(res["S"][n], beta[0, n] * np.outer(k[0, n], v[0, n]), atol=1e-14)
+        np.testing.assert_allclose(res["out"][0, n], 0.5 * beta[0, n] * np.dot(q[0, n], k[0, n]) * v[0, n], atol=1e-14)
+
+
+def test_units_are_independent_and_rows_are_keys():
+    """Swapping two units swaps their results; a decay on key channel 0 only touches state row 0."""
+    T, N, dk, dv = 3, 2, 3, 4
+    S0, q, k, v, lam, beta, bonus = rand_inputs(KDA, T, N, dk, dv)
+    a = oracle.eager_rollout(KDA, S0, q, k, v, lam, beta=beta)
+    b = oracle.eager_rollout(KDA, S0[::-1], q[:, ::-1], k[:, ::-1], v[:, ::-1], lam[:, ::-1], beta=beta[:, ::-1])
+    np.testing.assert_allclose(a["out"], b["out"][:, ::-1], atol=0)
+    lam1 = np.zeros((1, 1, dk)); lam1[0, 0, 0] = np.log(0.25)
+    res = oracle.eager_rollout(KDA, S0[:1], q[:1, :1], k[:1, :1], v[:1, :1], lam1, beta=np.zeros((1, 1)))
+    np.testing.assert_allclose(res["S"][0, 0], 0.25 * S0[0, 0], rtol=1e-15)
+    np.testing.assert_allclose(res["S"][0, 1:], S0[0, 1:], atol=0)
+
+
+def test_oracle_rejects_bad_arguments():
+    S0, q, k, v, lam, beta, bonus = rand_inputs(GDN, 2, 1, 2, 2)
+    with pytest.raises(ValueError):
+        oracle.eager_rollout(GDN, S0, q, k, v, lam)            # beta missing
+    with pytest.raises(ValueError):
+        oracle.eager_rollout(RWKV6, S0, q, k, v, np.zeros((2, 1, 2)))  # bonus missing
+    with pytest.raises(ValueError):
+        oracle.eager_rollout(GDN, S0, q[:1], k, v, lam, beta=beta)     # ragged T
+    with pytest.raises(ValueError):
+        oracle.eager_rollout(GDN, S0, q, k, v, lam, beta=beta, snapshot_at=[2, 1])
+    assert oracle.num_threads() >= 1
+
+
+# ---------------------------------------------------------------------------------------------
+# base-plus-log schedule (Algorithm 1, Eq. 4-6): closure under append and merge
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+@pytest.mark.parametrize("cap", [1, 2, 3, 5, 8])
+def test_log_schedule_equals_eager_after_every_append_and_merge(op, cap):
+    T, N, dk, dv = 11, 2, 4, 3
+    S0, q, k, v, lam, beta, bonus = rand_inputs(op, T, N, dk, dv)
+    ref = roll(op, S0, q, k, v, lam, beta, bonus, scale=1.3, snapshot_at=range(1, T + 1))
+    st = logical.LogState(op, S0, cap)
+    for t in range(T):
+        if (st.length == cap).all():
+            base_before = st.S_base.copy()
+            logical.merge(st, only_if_full=True)
+            assert (st.length == 0).all() and (st.lbar == 0).all()
+            assert not np.array_equal(base_before, st.S_base)
+            if t:  # the merge alone must not change the logical state
+                np.testing.assert_allclose(logical.materialize(st), ref["snapshots"][t - 1], atol=1e-12)
+        base_before = st.S_base.copy()
+        out = logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus, scale=1.3)
+        np.testing.assert_array_equal(st.S_base, base_before)      # append never writes the base
+        np.testing.assert_allclose(out, ref["out"][t], atol=1e-12)
+        np.testing.assert_allclose(logical.materialize(st), ref["snapshots"][t], atol=1e-12)
+        L = int(st.length[0])
+        np.testing.assert_allclose(st.U_log[:, L - 1], ref["b"][t], atol=1e-12)   # U entry = b_t
+        np.testing.assert_array_equal(st.K_log[:, L - 1], k[t])                    # K entry = a_t
+        # the newest snapshot is the running cumulative decay, so lbar need not be stored separately
+        np.testing.assert_array_equal(st.Lam_log[:, L - 1], st.lbar)
+        first = t - (L - 1)
+        np.testing.assert_allclose(st.Lam_log[:, L - 1], lam[first:t + 1].sum(axis=0).reshape(N, -1), atol=1e-13)
+
+
+def test_log_schedule_merge_variants():
+    op, cap, N, dk, dv = GDN, 4, 3, 3, 2
+    S0, q, k, v, lam, beta, bonus = rand_inputs(op, 6, N, dk, dv)
+    st = logical.LogState(op, S0, cap)
+    logical.merge(st)                                   # empty log: identity
+    np.testing.assert_array_equal(st.S_base, S0)
+    for t in range(2):
+        logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t])
+    logical.merge(st, only_if_full=True)                # not full: untouched
+    assert (st.length == 2).all()
+    np.testing.assert_array_equal(st.S_base, S0)
+    full = logical.materialize(st)
+    logical.merge(st)                                   # partial merge folds what is there
+    assert (st.length == 0).all()
+    np.testing.assert_allclose(st.S_base, full, atol=1e-14)
+    for t in range(2, 6):
+        logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t])
+    with pytest.raises(RuntimeError):
+        logical.decode_step(st, q[0], k[0], v[0], lam[0], beta=beta[0])
