@@ -1,0 +1,12 @@
+"""DeltaLog recurrent-state decode for linear attention on B200 (sm_100a).
+
+``binding``  ctypes binding of the C ABI in ``include/deltalog.h`` (the CUDA kernels live in ``csrc/``)
+``traffic``  the algorithmic-byte model of one decode cycle (Eq. 7-9 adapted to the split merge)
+``build``    compiles ``csrc/*.cu`` into ``libdeltalog.so``
+"""
+from . import traffic  # noqa: F401
+from .binding import (  # noqa: F401
+    BF16, F32, GDN, KDA, RWKV6, STATUS_BAD_SLOT, STATUS_LOG_FULL, STATUS_TIMEOUT, DeltalogError, Desc,
+    HostStaging, State, decode_step, decode_step_host, eager_step, launch_count, load_library, merge,
+    status_string, version,
+)

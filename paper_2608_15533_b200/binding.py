@@ -1,0 +1,240 @@
+"""ctypes binding of ``libdeltalog.so``: argument marshalling only.
+
+Every step of the decode / append / merge / eager path runs in the CUDA kernels behind the C ABI
+declared in ``include/deltalog.h``; this module turns torch tensors into raw pointers, passes the
+current CUDA stream and raises on a non-zero return code.  There is no CPU fallback: if the shared
+library is missing or cannot be loaded, importing the symbols raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+GDN, KDA, RWKV6 = 0, 1, 2
+F32, BF16 = 0, 1
+STATUS_LOG_FULL, STATUS_BAD_SLOT, STATUS_TIMEOUT = 1, 2, 4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAP_RANGE, ERR_CUDA = 0, 1, 2, 3, 4
+
+_TORCH_TO_DT = {torch.float32: F32, torch.bfloat16: BF16}
+_DT_TO_TORCH = {F32: torch.float32, BF16: torch.bfloat16}
+
+LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
+
+EXPORTS = (
+    "deltalog_decode_step", "deltalog_merge", "deltalog_eager_step", "deltalog_decode_step_host",
+    "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
+)
+
+
+class DeltalogError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (code {code})")
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("op", "num_slots", "H", "d_k", "d_v", "cap", "io_dtype", "klog_dtype", "ulog_dtype")] + \
+               [("scale", ctypes.c_float)]
+
+
+class _State(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("S_base", "K_log", "U_log", "decay_log", "log_len", "status")]
+
+
+class _Staging(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("q", "k", "v", "g", "beta", "out")]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load ``libdeltalog.so`` (built by ``paper_2608_15533_b200.build``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2608_15533_b200.build` "
+                "(there is no fallback path)")
+        lib = ctypes.CDLL(str(LIB_PATH))
+        vp, i32 = ctypes.c_void_p, ctypes.c_int32
+        lib.deltalog_decode_step.restype = ctypes.c_int
+        lib.deltalog_decode_step.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State)] + [vp] * 7 + [i32, vp, vp]
+        lib.deltalog_merge.restype = ctypes.c_int
+        lib.deltalog_merge.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State), vp, i32, i32, vp]
+        lib.deltalog_eager_step.restype = ctypes.c_int
+        lib.deltalog_eager_step.argtypes = [ctypes.POINTER(_Desc)] + [vp] * 8 + [i32, vp, vp, vp]
+        lib.deltalog_decode_step_host.restype = ctypes.c_int
+        lib.deltalog_decode_step_host.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State),
+                                                  ctypes.POINTER(_Staging)] + [vp] * 7 + [i32, vp, vp]
+        lib.deltalog_status_string.restype = ctypes.c_char_p
+        lib.deltalog_status_string.argtypes = [ctypes.c_int]
+        lib.deltalog_version.restype = ctypes.c_int
+        lib.deltalog_launch_count.restype = ctypes.c_uint64
+        _lib = lib
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return load_library().deltalog_status_string(int(code)).decode()
+
+
+def version() -> int:
+    return int(load_library().deltalog_version())
+
+
+def launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().deltalog_launch_count())
+
+
+@dataclass
+class Desc:
+    """Mirror of ``deltalog_desc``."""
+
+    op: int
+    num_slots: int
+    H: int
+    d_k: int
+    d_v: int
+    cap: int
+    io_dtype: int = BF16
+    klog_dtype: Optional[int] = None   # default: io_dtype
+    ulog_dtype: Optional[int] = None   # default: F32 for GDN / KDA, io_dtype for RWKV6
+    scale: float = 1.0
+
+    def __post_init__(self):
+        if self.klog_dtype is None:
+            self.klog_dtype = self.io_dtype
+        if self.ulog_dtype is None:
+            self.ulog_dtype = self.io_dtype if self.op == RWKV6 else F32
+
+    @property
+    def d_lambda(self) -> int:
+        return 1 if self.op == GDN else self.d_k
+
+    def c_struct(self) -> _Desc:
+        return _Desc(self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
+                     self.klog_dtype, self.ulog_dtype, float(self.scale))
+
+
+class State:
+    """Device tensors of the physical state (base, log, snapshots, lengths, status word)."""
+
+    def __init__(self, desc: Desc, S_base: torch.Tensor, device=None):
+        device = S_base.device if device is None else device
+        n, H, cap = desc.num_slots, desc.H, desc.cap
+        assert S_base.shape == (n, H, desc.d_k, desc.d_v) and S_base.dtype == torch.float32
+        self.desc = desc
+        self.S_base = S_base.contiguous()
+        self.K_log = torch.zeros(n, H, cap, desc.d_k, dtype=_DT_TO_TORCH[desc.klog_dtype], device=device)
+        self.U_log = torch.zeros(n, H, cap, desc.d_v, dtype=_DT_TO_TORCH[desc.ulog_dtype], device=device)
+        self.decay_log = torch.zeros(n, H, cap, desc.d_lambda, dtype=torch.float32, device=device)
+        self.log_len = torch.zeros(n, H, dtype=torch.int32, device=device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=device)
+
+    def c_struct(self) -> _State:
+        return _State(self.S_base.data_ptr(), self.K_log.data_ptr(), self.U_log.data_ptr(),
+                      self.decay_log.data_ptr(), self.log_len.data_ptr(), self.status.data_ptr())
+
+    def log_bytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.K_log, self.U_log, self.decay_log))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the C ABI must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise DeltalogError(rc, where)
+
+
+def decode_step(desc: Desc, state: State, q, k, v, g, beta=None, u_bonus=None, slot_idx=None, out=None,
+                stream=None) -> torch.Tensor:
+    """``deltalog_decode_step``: one token for ``B = q.shape[0]`` rows; returns ``out [B,H,d_v]``."""
+    B = q.shape[0]
+    if out is None:
+        out = torch.empty(B, desc.H, desc.d_v, dtype=q.dtype, device=q.device)
+    d, s = desc.c_struct(), state.c_struct()
+    rc = load_library().deltalog_decode_step(
+        ctypes.byref(d), ctypes.byref(s), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(u_bonus),
+        _ptr(slot_idx), B, _ptr(out), _stream(stream))
+    _check(rc, "deltalog_decode_step")
+    return out
+
+
+def merge(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None, only_if_full: bool = False,
+          stream=None) -> None:
+    """``deltalog_merge`` over the listed slots (all ``num_slots`` when ``slot_idx`` is None)."""
+    if n is None:
+        n = desc.num_slots if slot_idx is None else slot_idx.numel()
+    d, s = desc.c_struct(), state.c_struct()
+    rc = load_library().deltalog_merge(ctypes.byref(d), ctypes.byref(s), _ptr(slot_idx), int(n),
+                                       int(bool(only_if_full)), _stream(stream))
+    _check(rc, "deltalog_merge")
+
+
+def eager_step(desc: Desc, S: torch.Tensor, q, k, v, g, beta=None, u_bonus=None, slot_idx=None, out=None,
+               status=None, stream=None) -> torch.Tensor:
+    """``deltalog_eager_step``: the dense comparator; ``S`` is rewritten in place."""
+    B = q.shape[0]
+    if out is None:
+        out = torch.empty(B, desc.H, desc.d_v, dtype=q.dtype, device=q.device)
+    d = desc.c_struct()
+    rc = load_library().deltalog_eager_step(
+        ctypes.byref(d), _ptr(S), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(u_bonus),
+        _ptr(slot_idx), B, _ptr(out), _ptr(status), _stream(stream))
+    _check(rc, "deltalog_eager_step")
+    return out
+
+
+class HostStaging:
+    """Device staging buffers for ``decode_step_host`` (allocated once, reused every step)."""
+
+    def __init__(self, desc: Desc, B: int, device):
+        io = _DT_TO_TORCH[desc.io_dtype]
+        self.q = torch.empty(B, desc.H, desc.d_k, dtype=io, device=device)
+        self.k = torch.empty_like(self.q)
+        self.v = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
+        gshape = (B, desc.H) if desc.op == GDN else (B, desc.H, desc.d_k)
+        self.g = torch.empty(*gshape, dtype=torch.float32, device=device)
+        self.beta = torch.empty(B, desc.H, dtype=torch.float32, device=device)
+        self.out = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
+
+    def c_struct(self) -> _Staging:
+        return _Staging(*(t.data_ptr() for t in (self.q, self.k, self.v, self.g, self.beta, self.out)))
+
+    def h2d_bytes(self, desc: Desc) -> int:
+        ts = [self.q, self.k, self.v, self.g] + ([] if desc.op == RWKV6 else [self.beta])
+        return sum(t.numel() * t.element_size() for t in ts)
+
+    def d2h_bytes(self) -> int:
+        return self.out.numel() * self.out.element_size()
+
+
+def decode_step_host(desc: Desc, state: State, staging: HostStaging, host_q, host_k, host_v, host_g,
+                     host_beta, host_out, u_bonus=None, slot_idx=None, stream=None) -> None:
+    """``deltalog_decode_step_host``: token tensors and ``host_out`` are (pinned) host tensors."""
+    for t in (host_q, host_k, host_v, host_g, host_out):
+        assert t.device.type == "cpu"
+    B = host_q.shape[0]
+    d, s, st = desc.c_struct(), state.c_struct(), staging.c_struct()
+    rc = load_library().deltalog_decode_step_host(
+        ctypes.byref(d), ctypes.byref(s), ctypes.byref(st), _ptr(host_q), _ptr(host_k), _ptr(host_v),
+        _ptr(host_g), _ptr(host_beta), _ptr(u_bonus), _ptr(slot_idx), B, _ptr(host_out), _stream(stream))
+    _check(rc, "deltalog_decode_step_host")

@@ -1,0 +1,89 @@
+// Shared device helpers for the DeltaLog kernels: dtype conversion, cp.async staging, warp sums.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "deltalog.h"
+
+namespace deltalog {
+
+constexpr int kThreads = 256;  // every kernel in this library runs 256-thread CTAs
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxCap = 64;
+
+template <int DT> struct DType;
+template <> struct DType<DELTALOG_F32> { using type = float; };
+template <> struct DType<DELTALOG_BF16> { using type = __nv_bfloat16; };
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+    return __float2bfloat16_rn(x);
+}
+
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// Asynchronous 16-byte global -> shared copy (bypasses L1); both addresses 16-byte aligned.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
+
+// Cooperative async copy of `bytes` (multiple of 16) by the whole CTA.
+__device__ __forceinline__ void cta_cp_async(void *smem_dst, const void *gmem_src, int bytes, int tid) {
+    char *d = static_cast<char *>(smem_dst);
+    const char *s = static_cast<const char *>(gmem_src);
+    for (int off = tid * 16; off < bytes; off += kThreads * 16) cp_async16(d + off, s + off);
+}
+
+__device__ __forceinline__ float4 fma4(float a, const float4 &x, const float4 &acc) {
+    return make_float4(fmaf(a, x.x, acc.x), fmaf(a, x.y, acc.y), fmaf(a, x.z, acc.z), fmaf(a, x.w, acc.w));
+}
+
+// Resolve the pool slot of batch row b; returns false when the row must be skipped.
+__device__ __forceinline__ bool resolve_slot(const int32_t *slot_idx, int b, int num_slots, int32_t *status,
+                                             int tid, int &slot) {
+    slot = slot_idx ? slot_idx[b] : b;
+    if (slot < 0) return false;  // padding row
+    if (slot >= num_slots) {
+        if (tid == 0 && status) atomicOr(status, DELTALOG_STATUS_BAD_SLOT);
+        return false;
+    }
+    return true;
+}
+
+// Token-side arguments shared by the decode and eager kernels.
+struct TokenArgs {
+    const void *q, *k, *v;
+    const float *g, *beta, *u_bonus;
+    const int32_t *slot_idx;
+    void *out;
+    int32_t B;
+};
+
+struct StateArgs {
+    float *S_base;
+    void *K_log, *U_log;
+    float *decay_log;
+    int32_t *log_len;
+    int32_t *status;
+    int32_t num_slots, H, cap;
+    float scale;
+};
+
+}  // namespace deltalog

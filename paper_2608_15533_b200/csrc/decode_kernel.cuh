@@ -1,0 +1,193 @@
+// Decode + append kernel: one CTA per (batch row, head).
+//
+// Per unit (Algorithm 1, append branch; Eq. 4 and Eq. 6):
+//   lbar  = Lambda[len-1] (0 if the log is empty),  lbar' = lbar + lambda_t
+//   delta ops:  y_k = S_base^T (e^{lbar'} . k) + sum_i ck_i U_i,   ck_i = sum_j k_j e^{lbar'_j - Lambda_ij} K_ij
+//               y_q = S_base^T (e^{lbar'} . q) + sum_i cq_i U_i,   cq_i likewise with q
+//               b   = beta (v - y_k);   out = scale (y_q + (q.k) b)
+//   RWKV6:      y_r = S_base^T (e^{lbar} . r) + sum_i cr_i U_i  with the *old* lbar (pre-update readout)
+//               b   = v;                out = y_r + (r . (bonus . k)) v
+//   append:     K[len] = k, U[len] = b, Lambda[len] = lbar', len += 1.   S_base is never written.
+//
+// The 4*d_k*d_v bytes of the base tile are the only large read; they are requested first, as
+// 16-byte loads held in registers, before anything that depends on the (small) metadata.
+#pragma once
+
+#include "common.cuh"
+
+namespace deltalog {
+
+template <int D, typename IO, typename UL>
+constexpr size_t decode_smem_bytes(int op, int cap) {
+    const size_t dl = (op == DELTALOG_GDN) ? 1 : D;
+    size_t bytes = 0;
+    bytes += sizeof(float) * D * 5;                 // q, k (raw), mul_k, mul_q, lbar'/u scratch
+    bytes += sizeof(float) * D;                     // lbar_old (vector ops)
+    bytes += sizeof(float) * 2 * kMaxCap;           // replay coefficients
+    bytes += sizeof(float) * 2 * D * (kThreads / (D / 4));  // cross-row-lane partial sums
+    bytes += 16;                                    // scalars
+    bytes += sizeof(UL) * (size_t)cap * D;          // U log
+    bytes += sizeof(IO) * (size_t)cap * D;          // K log
+    bytes += sizeof(float) * (((size_t)cap * dl + 3) / 4 * 4);  // Lambda log
+    return bytes;
+}
+
+template <int OP, int D, typename IO, typename UL>
+__global__ void __launch_bounds__(kThreads, 2) decode_append_kernel(StateArgs st, TokenArgs tk) {
+    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
+    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr int DL = kVecDecay ? D : 1;
+    constexpr int C4 = D / 4;          // float4 columns per state row
+    constexpr int RL = kThreads / C4;  // rows covered by one pass of the CTA
+    constexpr int NP = D / RL;         // passes over the tile
+    constexpr int EPL = D / 32;        // key elements per lane in a warp-wide dot product
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    int slot;
+    if (!resolve_slot(tk.slot_idx, b, st.num_slots, st.status, tid, slot)) return;
+    const size_t unit = (size_t)slot * st.H + h;  // (slot, head) in the state pool
+    const size_t row = (size_t)b * st.H + h;      // (batch row, head) in the token tensors
+    const int cap = st.cap;
+
+    // ---- 1. request the whole base tile (independent of every other load) -------------------
+    const float4 *Sg = reinterpret_cast<const float4 *>(st.S_base + unit * D * D);
+    const int c4 = tid % C4, rl = tid / C4;
+    float4 s[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) s[p] = __ldg(Sg + (size_t)(p * RL + rl) * C4 + c4);
+
+    const int len = st.log_len[unit];
+    if (len >= cap) {  // Algorithm 1's else-branch is the caller's job (deltalog_merge)
+        if (tid == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
+        return;
+    }
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *q_s = reinterpret_cast<float *>(smem_raw);
+    float *k_s = q_s + D;
+    float *mk_s = k_s + D;      // e^{lbar'} . k
+    float *mq_s = mk_s + D;     // e^{lbar'} . q   (RWKV6: e^{lbar} . r)
+    float *b_s = mq_s + D;      // value-side factor, shared between the two output halves
+    float *lold_s = b_s + D;    // lbar (vector-decay ops)
+    float *ck_s = lold_s + D;   // [kMaxCap]
+    float *cq_s = ck_s + kMaxCap;
+    float *red_s = cq_s + kMaxCap;           // [RL][2][D]
+    float *scal_s = red_s + 2 * D * RL;      // [0] = q.k  (or r.(bonus.k))
+    UL *U_s = reinterpret_cast<UL *>(scal_s + 4);
+    IO *K_s = reinterpret_cast<IO *>(U_s + (size_t)cap * D);
+    float *Lam_s = reinterpret_cast<float *>(K_s + (size_t)cap * D);
+
+    // ---- 2. stage the live log entries (asynchronously) and the token vectors ---------------
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const float *Lg = st.decay_log + unit * cap * DL;
+    cta_cp_async(K_s, Kg, len * D * (int)sizeof(IO), tid);
+    cta_cp_async(U_s, Ug, len * D * (int)sizeof(UL), tid);
+    if (kVecDecay) cta_cp_async(Lam_s, Lg, len * D * (int)sizeof(float), tid);
+    cp_async_commit();
+    if (!kVecDecay && tid < len) Lam_s[tid] = Lg[tid];
+
+    const IO *qg = static_cast<const IO *>(tk.q) + row * D;
+    const IO *kg = static_cast<const IO *>(tk.k) + row * D;
+    const IO *vg = static_cast<const IO *>(tk.v) + row * D;
+    const float *gg = tk.g + row * DL;
+    IO k_raw = from_f32<IO>(0.f);
+    float lnew = 0.f;
+    if (tid < D) {
+        const float qv = to_f32(qg[tid]);
+        k_raw = kg[tid];
+        const float kv = to_f32(k_raw);
+        const float lold = (len > 0) ? Lg[(size_t)(len - 1) * DL + (kVecDecay ? tid : 0)] : 0.f;
+        lnew = lold + gg[kVecDecay ? tid : 0];
+        q_s[tid] = qv;
+        k_s[tid] = kv;
+        lold_s[tid] = kDelta ? lnew : lold;  // the decay level the replay coefficients refer to
+        const float e = expf(kDelta ? lnew : lold);
+        mk_s[tid] = e * kv;
+        mq_s[tid] = e * qv;
+    }
+    cp_async_wait_all();
+    __syncthreads();
+
+    // ---- 3. key-side replay coefficients: one warp per live entry ---------------------------
+    for (int i = warp; i < len; i += kWarps) {
+        float dq = 0.f, dk = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const int j = lane + 32 * e;
+            float kij = to_f32(K_s[i * D + j]);
+            if (kVecDecay) kij *= expf(lold_s[j] - Lam_s[i * D + j]);
+            dq = fmaf(q_s[j], kij, dq);
+            if (kDelta) dk = fmaf(k_s[j], kij, dk);
+        }
+        dq = warp_sum(dq);
+        if (kDelta) dk = warp_sum(dk);
+        if (lane == 0) {
+            const float w = kVecDecay ? 1.f : expf(lold_s[0] - Lam_s[i]);
+            cq_s[i] = w * dq;
+            if (kDelta) ck_s[i] = w * dk;
+        }
+    }
+    if (warp == kWarps - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
+        float d = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const int j = lane + 32 * e;
+            const float w = kDelta ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            d = fmaf(q_s[j] * w, k_s[j], d);
+        }
+        d = warp_sum(d);
+        if (lane == 0) scal_s[0] = d;
+    }
+
+    // ---- 4. base pass: two mat-vecs from one read of the tile -------------------------------
+    float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), aq = ak;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int r = p * RL + rl;
+        if (kDelta) ak = fma4(mk_s[r], s[p], ak);
+        aq = fma4(mq_s[r], s[p], aq);
+    }
+    float4 *red4 = reinterpret_cast<float4 *>(red_s);
+    if (kDelta) red4[(rl * 2 + 0) * C4 + c4] = ak;
+    red4[(rl * 2 + 1) * C4 + c4] = aq;
+    __syncthreads();
+
+    // ---- 5. reduce, replay the value-side log, form b and the output, append ----------------
+    const int which = tid / D, c = tid % D;  // which: 0 -> y_k half, 1 -> y_q half
+    float y = 0.f;
+    const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+    const int sel = kDelta ? which : 1;
+    if (active) {
+#pragma unroll
+        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+        const float *coef = sel ? cq_s : ck_s;
+        for (int i = 0; i < len; ++i) y = fmaf(coef[i], to_f32(U_s[i * D + c]), y);
+    }
+    UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
+    IO *og = static_cast<IO *>(tk.out) + row * D;
+    if (kDelta) {
+        if (tid < D) {
+            const float bval = tk.beta[row] * (to_f32(vg[c]) - y);
+            b_s[c] = bval;
+            Uout[c] = from_f32<UL>(bval);
+        }
+        __syncthreads();
+        if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
+    } else if (active) {
+        const IO v_raw = vg[c];
+        og[c] = from_f32<IO>(fmaf(scal_s[0], to_f32(v_raw), y));
+        Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+    }
+    if (tid < D) {
+        (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[tid] = k_raw;
+        if (kVecDecay) st.decay_log[(unit * cap + len) * DL + tid] = lnew;
+    }
+    if (tid == 0) {
+        if (!kVecDecay) st.decay_log[unit * cap + len] = lnew;
+        st.log_len[unit] = len + 1;
+    }
+}
+
+}  // namespace deltalog

@@ -1,0 +1,226 @@
+// C ABI of the DeltaLog decode library: host-side argument validation and kernel dispatch.
+// Declarations and the contract of every entry point are in include/deltalog.h.
+#include <atomic>
+#include <cstdint>
+#include <type_traits>
+
+#include "decode_kernel.cuh"
+#include "eager_kernel.cuh"
+#include "merge_kernel.cuh"
+
+namespace deltalog {
+namespace {
+
+std::atomic<uint64_t> g_launches{0};
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int validate_desc(const deltalog_desc *d) {
+    if (!d) return DELTALOG_ERR_INVALID_ARG;
+    if (d->op < DELTALOG_GDN || d->op > DELTALOG_RWKV6) return DELTALOG_ERR_INVALID_ARG;
+    if (d->num_slots <= 0 || d->H <= 0) return DELTALOG_ERR_INVALID_ARG;
+    if (d->io_dtype != DELTALOG_F32 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
+    if (d->klog_dtype != DELTALOG_F32 && d->klog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
+    if (d->ulog_dtype != DELTALOG_F32 && d->ulog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
+    if (d->d_k != d->d_v || (d->d_k != 64 && d->d_k != 128)) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
+    if (d->klog_dtype != d->io_dtype) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
+    const int want_u = (d->op == DELTALOG_RWKV6) ? d->io_dtype : (int)DELTALOG_F32;
+    if (d->ulog_dtype != want_u) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
+    if (d->cap < 1 || d->cap > kMaxCap) return DELTALOG_ERR_CAP_RANGE;
+    return DELTALOG_OK;
+}
+
+int validate_state(const deltalog_state *s) {
+    if (!s || !s->S_base || !s->K_log || !s->U_log || !s->decay_log || !s->log_len)
+        return DELTALOG_ERR_INVALID_ARG;
+    if (!aligned16(s->S_base) || !aligned16(s->K_log) || !aligned16(s->U_log) || !aligned16(s->decay_log))
+        return DELTALOG_ERR_INVALID_ARG;
+    return DELTALOG_OK;
+}
+
+int validate_token(const deltalog_desc *d, const void *q, const void *k, const void *v, const float *g,
+                   const float *beta, const float *u_bonus, int32_t B, const void *out) {
+    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
+    if (!q || !k || !v || !g || !out) return DELTALOG_ERR_INVALID_ARG;
+    if (d->op == DELTALOG_RWKV6 ? !u_bonus : !beta) return DELTALOG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(g))
+        return DELTALOG_ERR_INVALID_ARG;
+    return DELTALOG_OK;
+}
+
+StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
+    StateArgs a;
+    a.S_base = s->S_base;
+    a.K_log = s->K_log;
+    a.U_log = s->U_log;
+    a.decay_log = s->decay_log;
+    a.log_len = s->log_len;
+    a.status = s->status;
+    a.num_slots = d->num_slots;
+    a.H = d->H;
+    a.cap = d->cap;
+    a.scale = d->scale;
+    return a;
+}
+
+int finish_launch() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? DELTALOG_OK : DELTALOG_ERR_CUDA;
+}
+
+// Raise the dynamic shared-memory limit of a kernel once per process when it needs more than 48 KiB.
+template <typename K>
+int ensure_smem(K kernel, size_t bytes) {
+    if (bytes <= 48 * 1024) return DELTALOG_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        return DELTALOG_ERR_CUDA;
+    return DELTALOG_OK;
+}
+
+template <int OP, int D, typename IO>
+int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
+    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    auto kernel = decode_append_kernel<OP, D, IO, UL>;
+    const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
+    if (int rc = ensure_smem(kernel, smem)) return rc;
+    kernel<<<tk.B * st.H, kThreads, smem, stream>>>(st, tk);
+    return finish_launch();
+}
+
+template <int OP, int D, typename IO>
+int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
+                 cudaStream_t stream) {
+    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    auto kernel = merge_kernel<OP, D, IO, UL>;
+    const size_t smem = merge_smem_bytes<D>(st.cap);
+    if (int rc = ensure_smem(kernel, smem)) return rc;
+    kernel<<<n * st.H, kThreads, smem, stream>>>(st, slot_idx, only_if_full);
+    return finish_launch();
+}
+
+template <int OP, int D, typename IO>
+int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenArgs &tk, cudaStream_t stream) {
+    eager_step_kernel<OP, D, IO><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
+    return finish_launch();
+}
+
+// Expand (op, d, io dtype) into the template instantiation and call F<OP, D, IO>::run(args...).
+#define DELTALOG_DISPATCH(desc, CALL)                                                        \
+    do {                                                                                     \
+        const int op_ = (desc)->op, d_ = (desc)->d_k, io_ = (desc)->io_dtype;                \
+        if (op_ == DELTALOG_GDN) {                                                           \
+            DELTALOG_DISPATCH_D(DELTALOG_GDN, d_, io_, CALL);                                \
+        } else if (op_ == DELTALOG_KDA) {                                                    \
+            DELTALOG_DISPATCH_D(DELTALOG_KDA, d_, io_, CALL);                                \
+        } else {                                                                             \
+            DELTALOG_DISPATCH_D(DELTALOG_RWKV6, d_, io_, CALL);                              \
+        }                                                                                    \
+    } while (0)
+#define DELTALOG_DISPATCH_D(OP, d_, io_, CALL)                                               \
+    if (d_ == 64) {                                                                          \
+        if (io_ == DELTALOG_F32) { CALL(OP, 64, float); } else { CALL(OP, 64, __nv_bfloat16); } \
+    } else {                                                                                 \
+        if (io_ == DELTALOG_F32) { CALL(OP, 128, float); } else { CALL(OP, 128, __nv_bfloat16); } \
+    }
+
+}  // namespace
+}  // namespace deltalog
+
+using namespace deltalog;
+
+extern "C" {
+
+int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state, const void *q,
+                         const void *k, const void *v, const float *g, const float *beta,
+                         const float *u_bonus, const int32_t *slot_idx, int32_t B, void *out,
+                         void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
+    if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
+    if (B == 0) return DELTALOG_OK;
+    const StateArgs st = make_state_args(desc, state);
+    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define CALL_DECODE(OP, D, IO) return launch_decode<OP, D, IO>(st, tk, s)
+    DELTALOG_DISPATCH(desc, CALL_DECODE);
+#undef CALL_DECODE
+    return DELTALOG_ERR_INVALID_ARG;
+}
+
+int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const int32_t *slot_idx,
+                   int32_t n, int32_t only_if_full, void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
+    if (n < 0 || (!slot_idx && n > desc->num_slots)) return DELTALOG_ERR_INVALID_ARG;
+    if (n == 0) return DELTALOG_OK;
+    const StateArgs st = make_state_args(desc, state);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define CALL_MERGE(OP, D, IO) return launch_merge<OP, D, IO>(st, slot_idx, n, only_if_full, s)
+    DELTALOG_DISPATCH(desc, CALL_MERGE);
+#undef CALL_MERGE
+    return DELTALOG_ERR_INVALID_ARG;
+}
+
+int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, const void *k,
+                        const void *v, const float *g, const float *beta, const float *u_bonus,
+                        const int32_t *slot_idx, int32_t B, void *out, int32_t *status, void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (!S || !aligned16(S)) return DELTALOG_ERR_INVALID_ARG;
+    if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
+    if (B == 0) return DELTALOG_OK;
+    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define CALL_EAGER(OP, D, IO) return launch_eager<OP, D, IO>(S, desc, status, tk, s)
+    DELTALOG_DISPATCH(desc, CALL_EAGER);
+#undef CALL_EAGER
+    return DELTALOG_ERR_INVALID_ARG;
+}
+
+int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *state,
+                              const deltalog_staging *staging, const void *host_q,
+                              const void *host_k, const void *host_v, const float *host_g,
+                              const float *host_beta, const float *u_bonus,
+                              const int32_t *slot_idx, int32_t B, void *host_out, void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (!staging || !host_q || !host_k || !host_v || !host_g || !host_out) return DELTALOG_ERR_INVALID_ARG;
+    if (desc->op != DELTALOG_RWKV6 && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
+    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
+    if (B == 0) return DELTALOG_OK;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t units = (size_t)B * desc->H;
+    const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
+    const size_t vec = units * desc->d_k * esz;
+    const size_t gbytes = units * (desc->op == DELTALOG_GDN ? 1 : desc->d_k) * sizeof(float);
+    if (!staging->q || !staging->k || !staging->v || !staging->g || !staging->out) return DELTALOG_ERR_INVALID_ARG;
+    bool ok = cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (desc->op != DELTALOG_RWKV6)
+        ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s) ==
+                       cudaSuccess;
+    if (!ok) return DELTALOG_ERR_CUDA;
+    if (int rc = deltalog_decode_step(desc, state, staging->q, staging->k, staging->v, staging->g,
+                                      staging->beta, u_bonus, slot_idx, B, staging->out, stream))
+        return rc;
+    if (cudaMemcpyAsync(host_out, staging->out, units * desc->d_v * esz, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return DELTALOG_ERR_CUDA;
+    return DELTALOG_OK;
+}
+
+const char *deltalog_status_string(int code) {
+    switch (code) {
+        case DELTALOG_OK: return "ok";
+        case DELTALOG_ERR_INVALID_ARG: return "invalid argument (null / misaligned pointer, bad enum or negative count)";
+        case DELTALOG_ERR_UNSUPPORTED_SHAPE: return "unsupported shape or dtype combination";
+        case DELTALOG_ERR_CAP_RANGE: return "log capacity outside 1..64";
+        case DELTALOG_ERR_CUDA: return "CUDA runtime error";
+        default: return "unknown status code";
+    }
+}
+
+int deltalog_version(void) { return 100; }
+
+uint64_t deltalog_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

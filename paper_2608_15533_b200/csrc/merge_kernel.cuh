@@ -1,0 +1,84 @@
+// Merge kernel: one CTA per (listed slot, head) folds the live log into the dense base with a
+// single read and a single write of the tile (Eq. 5 without the current-token term):
+//
+//   S_base[j, :] <- e^{lbar_j} S_base[j, :] + sum_{i<len} (e^{lbar_j - Lambda_ij} K_ij) U_i[:],   len <- 0
+//
+// with lbar = Lambda[len-1].  The key-side weights A_ij = e^{lbar_j - Lambda_ij} K_ij are formed
+// once in shared memory; every thread then owns NP consecutive rows x 4 columns of the tile and
+// applies the rank-len update to them in registers.
+#pragma once
+
+#include "common.cuh"
+
+namespace deltalog {
+
+template <int D>
+constexpr size_t merge_smem_bytes(int cap) {
+    return sizeof(float) * ((size_t)2 * cap * D + D);  // A [cap][D], U [cap][D] (fp32), e^{lbar} [D]
+}
+
+template <int OP, int D, typename IO, typename UL>
+__global__ void __launch_bounds__(kThreads, 2)
+merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full) {
+    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr int DL = kVecDecay ? D : 1;
+    constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL;
+
+    const int tid = threadIdx.x;
+    const int n = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    int slot;
+    if (!resolve_slot(slot_idx, n, st.num_slots, st.status, tid, slot)) return;
+    const size_t unit = (size_t)slot * st.H + h;
+    const int cap = st.cap;
+    const int len = st.log_len[unit];
+    if (len <= 0 || len > cap || (only_if_full && len < cap)) return;  // nothing to fold: no dense write
+
+    // each thread owns rows [rl*NP, rl*NP + NP) x columns [4*c4, 4*c4 + 4)
+    float4 *Sg = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
+    const int c4 = tid % C4, rl = tid / C4;
+    float4 s[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) s[p] = Sg[(size_t)(rl * NP + p) * C4 + c4];
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][D]
+    float *U_s = A_s + (size_t)cap * D;                // [len][D]
+    float *e_s = U_s + (size_t)cap * D;                // [D]
+
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const float *Lg = st.decay_log + unit * cap * DL;
+    const float *lbar = Lg + (size_t)(len - 1) * DL;
+    for (int x = tid; x < len * D; x += kThreads) {
+        const int i = x / D, j = x % D;
+        const float w = expf(kVecDecay ? (lbar[j] - Lg[(size_t)i * D + j]) : (lbar[0] - Lg[i]));
+        A_s[x] = w * to_f32(Kg[x]);
+        U_s[x] = to_f32(Ug[x]);
+    }
+    if (tid < D) e_s[tid] = expf(lbar[kVecDecay ? tid : 0]);
+    __syncthreads();
+
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const float e = e_s[rl * NP + p];
+        s[p] = make_float4(e * s[p].x, e * s[p].y, e * s[p].z, e * s[p].w);
+    }
+    const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
+    for (int i = 0; i < len; ++i) {
+        const float4 u = U4[i * C4 + c4];
+        const float4 *a4 = reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP);
+#pragma unroll
+        for (int p4 = 0; p4 < NP / 4; ++p4) {
+            const float4 a = a4[p4];
+            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
+            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
+            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
+            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < NP; ++p) Sg[(size_t)(rl * NP + p) * C4 + c4] = s[p];
+    if (tid == 0) st.log_len[unit] = 0;
+}
+
+}  // namespace deltalog
