@@ -1,0 +1,413 @@
+#!/usr/bin/env python
+"""Benchmark of the DeltaLog decode hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..4] [--cap C] [--impl ours|reference]
+
+One "step" is one decode token for the whole batch of the workload: the decode+append kernel, and
+the merge kernel whenever the logs are full (every ``cap`` steps), i.e. the complete hot path.
+Rank 0 prints ONE JSON line.  ``value`` is (sequence*head) state updates per second with all inputs
+resident in HBM; ``e2e`` is the same metric through ``deltalog_decode_step_host`` with the token
+tensors in pinned host memory and the output read back to the host every step.
+
+With N > 1 (one process per GPU, launched by ``torch.distributed.run``) every rank decodes its own
+shard of batch rows -- the path has no exchange step -- and the time is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+import torch  # noqa: E402
+
+import workloads  # noqa: E402
+from paper_2608_15533_b200 import launch, traffic  # noqa: E402
+
+METRIC = "state-update (seq*head)-steps/s"
+UNIT = "(seq*head)-steps/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
+# captures summarised under profiles/ (bytes per (sequence, head) unit; None = not captured).
+NCU_DECODE_TRAFFIC_PER_UNIT = {}
+
+
+def measured_peak_gbs():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows, self.proc, self.gpu = [], None, gpu_index
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, flag in zip(names, r[3:7]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def unit_shape(wl: workloads.Workload) -> traffic.UnitShape:
+    io = 4 if wl.io_dtype == torch.float32 else 2
+    ul = io if wl.op == workloads.RWKV6 else 4
+    return traffic.UnitShape(wl.op, wl.d, wl.d, io_bytes=io, klog_bytes=io, ulog_bytes=ul)
+
+
+class Rig:
+    """Device-resident state and a ring of pre-generated token batches for one workload / capacity."""
+
+    RING = 8
+
+    def __init__(self, wl, cap, device, seed_offset=0, layers=1):
+        import paper_2608_15533_b200 as dl
+
+        self.dl, self.wl, self.cap, self.device, self.layers = dl, wl, cap, device, layers
+        io = dl.F32 if wl.io_dtype == torch.float32 else dl.BF16
+        self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io)
+        self.states, self.rings, self.bonus = [], [], []
+        for layer in range(layers):
+            src = workloads.TokenSource(wl, device=device, seed=wl.seed + 1000 * seed_offset + layer)
+            self.states.append(dl.State(self.desc, src.initial_state()))
+            self.bonus.append(src.bonus())
+            self.rings.append([src.token() for _ in range(self.RING)])
+        self.out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
+        self.slot_idx = None
+        self.step_slots = None   # optional per-step slot lists (staggered start)
+
+    def decode(self, t, layer=0, slot_idx=None):
+        tok = self.rings[layer][t % self.RING]
+        self.dl.decode_step(self.desc, self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
+                            beta=tok["beta"], u_bonus=self.bonus[layer],
+                            slot_idx=self.slot_idx if slot_idx is None else slot_idx, out=self.out)
+
+    def merge(self, layer=0, only_if_full=True):
+        self.dl.merge(self.desc, self.states[layer], slot_idx=self.slot_idx, n=self.wl.batch,
+                      only_if_full=only_if_full)
+
+    def reset_logs(self):
+        for layer in range(self.layers):
+            self.merge(layer, only_if_full=False)
+
+    def status(self):
+        return [int(s.status.item()) for s in self.states]
+
+
+def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
+    """Time exactly ``steps`` steps (decode every step, merge after every cap-th) on the current
+    stream; returns total ms, summed decode-kernel ms and summed merge-kernel ms."""
+    cap = rig.cap
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    start, end = ev(), ev()
+    d0 = [ev() for _ in range(steps)] if per_kernel else None
+    d1 = [ev() for _ in range(steps)] if per_kernel else None
+    m1 = {}
+    launch.barrier()
+    torch.cuda.synchronize()
+    start.record()
+    for t in range(steps):
+        for layer in range(rig.layers):
+            if per_kernel and layer == 0:
+                d0[t].record()
+            rig.decode(t, layer)
+            if per_kernel and layer == 0:
+                d1[t].record()
+            if (t + 1) % cap == 0:
+                rig.merge(layer)
+                if per_kernel and layer == 0:
+                    m1[t] = ev(); m1[t].record()
+    end.record()
+    torch.cuda.synchronize()
+    launch.barrier()
+    total = start.elapsed_time(end)
+    dec = sum(a.elapsed_time(b) for a, b in zip(d0, d1)) if per_kernel else None
+    mrg = sum(d1[t].elapsed_time(e) for t, e in m1.items()) if per_kernel else None
+    return total, dec, mrg, len(m1)
+
+
+def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int):
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dl = rig.dl
+    torch.cuda.synchronize()
+    start.record()
+    for t in range(steps):
+        tok = rig.rings[0][t % rig.RING]
+        dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                      u_bonus=rig.bonus[0], out=rig.out)
+    end.record()
+    torch.cuda.synchronize()
+    return start.elapsed_time(end)
+
+
+def time_e2e_loop(rig: Rig, steps: int):
+    """The same cycle through the host-buffer entry point: every step copies q, k, v, g, beta from
+    pinned host memory and reads the output back to pinned host memory."""
+    dl, wl = rig.dl, rig.wl
+    staging = dl.HostStaging(rig.desc, wl.batch, rig.device)
+    host_ring = [{k: (v.cpu().pin_memory() if v is not None else None) for k, v in tok.items()}
+                 for tok in rig.rings[0]]
+    host_out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()
+    rig.reset_logs()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def run(n):
+        for t in range(n):
+            tok = host_ring[t % rig.RING]
+            dl.decode_step_host(rig.desc, rig.states[0], staging, tok["q"], tok["k"], tok["v"], tok["g"],
+                                tok["beta"], host_out, u_bonus=rig.bonus[0], slot_idx=rig.slot_idx)
+            if (t + 1) % rig.cap == 0:
+                rig.merge(0)
+
+    run(rig.cap)  # warm the copy path, ends on a merge
+    launch.barrier()
+    torch.cuda.synchronize()
+    start.record()
+    run(steps)
+    end.record()
+    torch.cuda.synchronize()
+    launch.barrier()
+    return start.elapsed_time(end), staging.h2d_bytes(rig.desc), staging.d2h_bytes()
+
+
+def cpu_baseline(wl, units: int, steps: int):
+    """Time the fp64 oracle, as it stands, on a bounded sample of the workload's units."""
+    import numpy as np
+
+    import oracle
+
+    small = wl.scaled(batch=max(1, units // wl.H), num_slots=None)
+    src = workloads.TokenSource(small, device="cpu")
+    S0 = src.initial_state().double().numpy().reshape(-1, wl.d, wl.d)
+    bonus = src.bonus()
+    N = S0.shape[0]
+    toks = [src.token() for _ in range(steps)]
+    f = lambda key: np.stack([t[key].double().numpy().reshape(N, -1) for t in toks])
+    q, k, v, g = f("q"), f("k"), f("v"), f("g")
+    beta = f("beta")[..., 0] if wl.op != workloads.RWKV6 else None
+    bon = np.tile(bonus.double().numpy(), (small.batch, 1)) if bonus is not None else None
+    t0 = time.perf_counter()
+    oracle.eager_rollout(wl.op, S0, q, k, v, g, beta=beta, bonus=bon)
+    dt = time.perf_counter() - t0
+    return {"value": N * steps / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{N} (seq*head) units x {steps} tokens of {wl.name}, fp64 eager recurrence, {dt:.2f} s"}, dt
+
+
+def run_reference(args, wl):
+    """``--impl reference``: the CPU oracle timed on the host cores (rank 0 only)."""
+    rank, size, _ = launch.world()
+    if rank != 0:
+        return
+    units = 512
+    base, dt = cpu_baseline(wl, units, max(args.steps, 1))
+    n_units = max(1, units // wl.H) * wl.H
+    line = {
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "sample_units_per_step": n_units,
+                   "note": "each step is one token over a bounded sample of the workload's units on the host"},
+        "cpu_baseline": {**base},
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=32)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--cap", type=int, default=16, help="log capacity of the headline number")
+    ap.add_argument("--no-extras", action="store_true", help="skip the capacity sweep, eager and CPU legs")
+    ap.add_argument("--only-hot-loop", action="store_true",
+                    help="warm-up and timed loop only (for profiler captures)")
+    args = ap.parse_args()
+    wl = workloads.CONFIGS[args.config]
+    if args.impl == "reference":
+        return run_reference(args, wl)
+
+    rank, size, local = launch.init("nccl")
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    import paper_2608_15533_b200 as dl
+
+    cap = args.cap
+    warmup = max(args.warmup, 3)
+    layers = wl.layers
+    rig = Rig(wl, cap, device, seed_offset=rank, layers=layers)
+    if wl.staggered:
+        rig.slot_idx = workloads.slot_permutation(wl).to(device)
+    u = unit_shape(wl)
+    units = wl.units
+
+    # ---- warm-up, then the timed region: exactly K steps ---------------------------------------
+    launches0 = dl.launch_count()
+    for t in range(warmup):
+        for layer in range(layers):
+            rig.decode(t, layer)
+            if (t + 1) % cap == 0:
+                rig.merge(layer)
+    rig.reset_logs()
+    torch.cuda.synchronize()
+    warm_launches = dl.launch_count() - launches0
+    if args.only_hot_loop:
+        time_cycle_loop(rig, args.steps, per_kernel=False)
+        return launch.finalize()
+    with ClockSampler(local) as clocks:
+        l0 = dl.launch_count()
+        total_ms, dec_ms, mrg_ms, n_merges = time_cycle_loop(rig, args.steps)
+        gpu_launches = dl.launch_count() - l0
+    assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
+    total_ms = launch.max_over_ranks(total_ms, device)
+    all_units = launch.sum_over_ranks(units * layers, device)
+    ms_per_step = total_ms / args.steps
+    value = all_units * args.steps / (total_ms * 1e-3)
+
+    cyc = traffic.cycle_bytes(u, cap)
+    peak, peak_kind = measured_peak_gbs()
+    fills = [t % cap for t in range(args.steps)]
+    dec_bytes = statistics.mean(traffic.decode_read(u, f) + traffic.decode_write(u) for f in fills) * units
+    dec_ms_avg = dec_ms / args.steps
+    achieved = dec_bytes / (dec_ms_avg * 1e-3) / 1e9
+    traffic_ncu = NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
+            "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
+            "io": str(wl.io_dtype).replace("torch.", ""), "merge": f"after every {cap}th step",
+            "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
+            "parallelism": f"rows sharded over {size} GPU(s), no collective",
+        },
+        "clocks": clocks.summary(),
+        "gpu_launches": gpu_launches,
+        "roofline": {
+            "bound": "hbm", "kernel": "decode_append_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic_ncu * units if traffic_ncu else None,
+            "algorithmic_bytes_per_launch": dec_bytes, "avg_launch_ms": dec_ms_avg,
+            "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+        },
+        "amortized": {
+            "algorithmic_bytes_per_unit_step": cyc["total"],
+            "hbm_gbs": cyc["total"] * all_units / (ms_per_step * 1e-3) / 1e9,
+            "bytes_written_per_unit_step": cyc["write"], "write_reduction_vs_eager": cyc["write_reduction"],
+            "decode_ms_per_step": dec_ms_avg, "merge_ms_per_merge": (mrg_ms / n_merges) if n_merges else None,
+        },
+    }
+    line["amortized"]["frac_of_nominal_8TBs"] = line["amortized"]["hbm_gbs"] / NOMINAL_HBM_GBS / size
+    line["amortized"]["frac_of_measured"] = line["amortized"]["hbm_gbs"] / peak / size
+
+    # ---- end-to-end leg: token tensors from pinned host memory, output back to the host --------
+    e2e_ms, h2d, d2h = time_e2e_loop(rig, args.steps)
+    e2e_ms = launch.max_over_ranks(e2e_ms, device)
+    e2e_units = launch.sum_over_ranks(units, device)
+    line["e2e"] = {"value": e2e_units * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps,
+                   "note": "state stays resident; q,k,v,g,beta in and out back every step, layer 0"}
+
+    if not args.no_extras and rank == 0:
+        # eager dense comparator on the same inputs
+        rig.reset_logs()
+        S = rig.states[0].S_base
+        time_eager_loop(rig, S, 8)
+        eager_ms = time_eager_loop(rig, S, args.steps) / args.steps
+        eager_bytes = (traffic.eager_read(u) + traffic.eager_write(u)) * units
+        line["eager_kernel"] = {"ms_per_step": eager_ms, "value": units / (eager_ms * 1e-3),
+                                "hbm_gbs": eager_bytes / (eager_ms * 1e-3) / 1e9,
+                                "bytes_written_per_unit_step": traffic.eager_write(u)}
+        line["speedup_vs_eager_kernel"] = eager_ms / (ms_per_step / layers)
+        sweep = {}
+        for c in wl.caps:
+            if c == cap and layers == 1:
+                sweep[str(c)] = {"ms_per_step": ms_per_step, "value": value,
+                                 "write_reduction_vs_eager": cyc["write_reduction"],
+                                 "hbm_gbs": line["amortized"]["hbm_gbs"]}
+                continue
+            if layers > 1:
+                continue
+            del rig
+            torch.cuda.empty_cache()
+            rig = Rig(wl, c, device, seed_offset=rank)
+            for t in range(max(c, 3)):
+                rig.decode(t);
+                if (t + 1) % c == 0:
+                    rig.merge()
+            rig.reset_logs()
+            ms, _, _, _ = time_cycle_loop(rig, args.steps, per_kernel=False)
+            cc = traffic.cycle_bytes(u, c)
+            sweep[str(c)] = {"ms_per_step": ms / args.steps, "value": units * args.steps / (ms * 1e-3),
+                             "write_reduction_vs_eager": cc["write_reduction"],
+                             "hbm_gbs": cc["total"] * units / (ms / args.steps * 1e-3) / 1e9}
+        line["capacity_sweep"] = sweep
+        small = wl.scaled(layers=1)
+        line["cpu_baseline"], _ = cpu_baseline(small, 2048, 128)
+    if rank == 0:
+        print(json.dumps(line))
+    launch.finalize()
+
+
+if __name__ == "__main__":
+    main()

@@ -119,8 +119,13 @@ class Desc:
         return 1 if self.op == GDN else self.d_k
 
     def c_struct(self) -> _Desc:
-        return _Desc(self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
-                     self.klog_dtype, self.ulog_dtype, float(self.scale))
+        key = (self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
+               self.klog_dtype, self.ulog_dtype, float(self.scale))
+        cached = self.__dict__.get("_c")
+        if cached is None or cached[0] != key:
+            cached = (key, _Desc(*key))
+            self.__dict__["_c"] = cached
+        return cached[1]
 
 
 class State:
@@ -139,8 +144,13 @@ class State:
         self.status = torch.zeros(1, dtype=torch.int32, device=device)
 
     def c_struct(self) -> _State:
-        return _State(self.S_base.data_ptr(), self.K_log.data_ptr(), self.U_log.data_ptr(),
-                      self.decay_log.data_ptr(), self.log_len.data_ptr(), self.status.data_ptr())
+        ptrs = (self.S_base.data_ptr(), self.K_log.data_ptr(), self.U_log.data_ptr(),
+                self.decay_log.data_ptr(), self.log_len.data_ptr(), self.status.data_ptr())
+        cached = getattr(self, "_c", None)
+        if cached is None or cached[0] != ptrs:
+            cached = (ptrs, _State(*ptrs))
+            self._c = cached
+        return cached[1]
 
     def log_bytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.K_log, self.U_log, self.decay_log))
