@@ -26,6 +26,31 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
     return __float2bfloat16_rn(x);
 }
 
+// Load N (2 or 4) consecutive elements as one vector access and widen them to fp32.
+template <typename T, int N>
+__device__ __forceinline__ void load_vec(const T *p, float (&out)[N]);
+template <>
+__device__ __forceinline__ void load_vec<float, 4>(const float *p, float (&out)[4]) {
+    const float4 v = *reinterpret_cast<const float4 *>(p);
+    out[0] = v.x, out[1] = v.y, out[2] = v.z, out[3] = v.w;
+}
+template <>
+__device__ __forceinline__ void load_vec<float, 2>(const float *p, float (&out)[2]) {
+    const float2 v = *reinterpret_cast<const float2 *>(p);
+    out[0] = v.x, out[1] = v.y;
+}
+template <>
+__device__ __forceinline__ void load_vec<__nv_bfloat16, 4>(const __nv_bfloat16 *p, float (&out)[4]) {
+    const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    out[0] = __uint_as_float(v.x << 16), out[1] = __uint_as_float(v.x & 0xffff0000u);
+    out[2] = __uint_as_float(v.y << 16), out[3] = __uint_as_float(v.y & 0xffff0000u);
+}
+template <>
+__device__ __forceinline__ void load_vec<__nv_bfloat16, 2>(const __nv_bfloat16 *p, float (&out)[2]) {
+    const uint32_t v = *reinterpret_cast<const uint32_t *>(p);
+    out[0] = __uint_as_float(v << 16), out[1] = __uint_as_float(v & 0xffff0000u);
+}
+
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);

@@ -1,0 +1,583 @@
+// Persistent, warp-specialised decode + append kernel.
+//
+// Same arithmetic as decode_append_kernel (Algorithm 1, append branch; Eq. 4 and Eq. 6), different
+// schedule.  One CTA stays resident per SM and walks over its share of the (batch row, head) units.
+// Four roles run concurrently and hand work to one another through mbarriers:
+//
+//   base producer (1 warp)  bulk asynchronous copies (cp.async.bulk) of 16 KiB chunks of the fp32
+//                           base tile (d=128: 4 chunks per unit, d=64: 1) into the base ring;
+//   aux producer  (1 warp)  per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
+//                           token vectors q, k, v (and g, bonus where they are vectors) and a small
+//                           metadata record (len, flags, scalar gate, beta) into the aux ring;
+//   stream group  (8 warps) the base pass only: the two mat-vecs S_base^T (e^lbar . k) and
+//                           S_base^T (e^lbar . q) from each chunk the moment it lands, releasing the
+//                           chunk at once, so the HBM stream never waits for a unit's epilogue;
+//   scalar group  (8 warps) everything that does not touch the base: for unit i+1 the cumulative
+//                           decay, the decayed multipliers and the key-side replay coefficients
+//                           (the paper's ReplayPrep, here a pipeline stage instead of a launch); for
+//                           unit i the cross-warp reduction, the value-side replay, b, the output and
+//                           the append.
+//
+// No compute warp ever issues a global load; what the scalar group writes (out, the appended entry
+// and the new length) is fire-and-forget.  Every wait on an mbarrier is bounded in time: when it
+// gives up it raises the CTA's abort flag, ORs DELTALOG_STATUS_TIMEOUT into the status word, and all
+// roles leave their loops; the producers then wait (bounded again) for the copies they still have
+// in flight before the CTA exits.
+#pragma once
+
+#include "common.cuh"
+
+namespace deltalog {
+
+constexpr int kChunkBytes = 16384;
+constexpr int kPipeConsumers = 256;                    // threads of the stream group and of the scalar group
+constexpr int kPipeThreads = 2 * kPipeConsumers + 64;  // + base-ring producer warp + aux-ring producer warp
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+enum : int { kMetaSkip = 1, kMetaFull = 2 };
+
+__host__ __device__ constexpr int align_up(int x, int a) { return (x + a - 1) / a * a; }
+
+// Byte offsets inside one aux-ring stage (all multiples of 16).
+template <int OP, int D, typename IO, typename UL>
+struct AuxLayout {
+    static constexpr bool kVec = (OP != DELTALOG_GDN);
+    static constexpr int DL = kVec ? D : 1;
+    int K, U, L, q, k, v, g, bonus, meta, bytes;
+    __host__ __device__ explicit AuxLayout(int cap) {
+        K = 0;
+        U = K + cap * D * (int)sizeof(IO);
+        L = U + cap * D * (int)sizeof(UL);
+        q = L + align_up(cap * DL * 4, 16);
+        k = q + D * (int)sizeof(IO);
+        v = k + D * (int)sizeof(IO);
+        g = v + D * (int)sizeof(IO);
+        bonus = g + (kVec ? D * 4 : 0);
+        meta = bonus + (OP == DELTALOG_RWKV6 ? D * 4 : 0);
+        bytes = align_up(meta + 32, 128);
+    }
+};
+
+// Hand-over buffer between the roles, two slots (unit i and unit i+1 are in flight together).
+// Per slot (floats): q, k, mul_k, mul_q, lbar, lbar', b [7*D], ck, cq [2*64], scalars [4]: q.k and the
+// unit's flags; then the stream group's partial sums [RL][2][D].
+template <int D>
+__host__ __device__ constexpr int pipe_slot_floats() {
+    return 7 * D + 2 * kMaxCap + 4 + 2 * D * (kPipeConsumers / (D / 4));
+}
+template <int D>
+__host__ __device__ constexpr int pipe_scratch_bytes() {
+    return 2 * align_up(pipe_slot_floats<D>() * 4, 128);
+}
+constexpr int kPipeBarrierBytes = 1024;  // mbarriers (2 x 32 + 2 x 8 + 4 at most) and the abort flags
+
+struct PipeCfg {
+    int n_base;  // stages of the base ring
+    int n_aux;   // stages of the aux ring
+};
+
+template <int OP, int D, typename IO, typename UL>
+__host__ inline int pipe_smem_bytes(int cap, PipeCfg cfg) {
+    return kPipeBarrierBytes + pipe_scratch_bytes<D>() + cfg.n_aux * AuxLayout<OP, D, IO, UL>(cap).bytes +
+           cfg.n_base * kChunkBytes;
+}
+
+// ---- mbarrier / bulk-copy primitives ---------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bulk asynchronous copy global -> this CTA's shared memory; bytes % 16 == 0, both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
+    return t;
+}
+
+// Wait for a phase of an mbarrier, giving up after kWaitLimitNs or as soon as the CTA aborts.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+// OR-reduction of a predicate over the consumer warps (named barrier 1), also a consumer-only barrier.
+__device__ __forceinline__ bool consumers_any(bool pred) {
+    uint32_t res;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, 1, %2, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(res)
+        : "r"((uint32_t)pred), "n"(kPipeConsumers)
+        : "memory");
+    return res != 0;
+}
+__device__ __forceinline__ void consumers_sync() {
+    asm volatile("bar.sync 1, %0;\n" ::"n"(kPipeConsumers) : "memory");
+}
+
+struct RingPos {  // position in a ring of n stages: stage index and phase parity
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance(int n) {
+        if (++stage == n) {
+            stage = 0;
+            phase ^= 1u;
+        }
+    }
+};
+
+template <int OP, int D, typename IO, typename UL>
+__global__ void __launch_bounds__(kPipeThreads, 1)
+decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
+    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
+    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr int DL = kVecDecay ? D : 1;
+    constexpr int C4 = D / 4;
+    constexpr int RL = kPipeConsumers / C4;          // row groups of the stream group
+    constexpr int NCHUNK = D * D * 4 / kChunkBytes;  // chunks per base tile
+    constexpr int CH_ROWS = D / NCHUNK;              // rows per chunk
+    constexpr int PPC = CH_ROWS / RL;                // rows of a chunk per stream thread
+    static_assert(PPC == 4, "the base pass is written for four rows per thread and chunk");
+    constexpr int EPL = D / 32;                      // key channels per lane in the coefficient phase
+    constexpr int kGroupWarps = kPipeConsumers / 32;
+    constexpr int SLOT = align_up(pipe_slot_floats<D>() * 4, 128) / 4;  // floats per hand-over slot
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    const AuxLayout<OP, D, IO, UL> lay(st.cap);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kPipeBarrierBytes - 16);
+    float *scratch = reinterpret_cast<float *>(smem + kPipeBarrierBytes);
+    unsigned char *aux_ring = smem + kPipeBarrierBytes + pipe_scratch_bytes<D>();
+    unsigned char *base_ring = aux_ring + (size_t)cfg.n_aux * lay.bytes;
+
+    const int NB = cfg.n_base, NA = cfg.n_aux;
+    const uint32_t full_base = smem_addr(bars), empty_base = full_base + 8u * NB;
+    const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * NA;
+    const uint32_t prep_done = empty_aux + 8u * NA;   // [2] scalar group -> stream group: multipliers ready
+    const uint32_t stream_done = prep_done + 16u;     // [2] stream group -> scalar group: partial sums ready
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) {
+        for (int i = 0; i < NB; ++i) {
+            mbar_init(full_base + 8u * i, 1);
+            mbar_init(empty_base + 8u * i, kGroupWarps);
+        }
+        for (int i = 0; i < NA; ++i) {
+            mbar_init(full_aux + 8u * i, 1);
+            mbar_init(empty_aux + 8u * i, kGroupWarps);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(prep_done + 8u * i, 1);
+            mbar_init(stream_done + 8u * i, kGroupWarps);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;  // separate flag for the drain waits after an abort
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+    }
+    __syncthreads();
+
+    const int total = tk.B * st.H;
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_items = (total - first + stride - 1) / stride;
+    const int cap = st.cap, H = st.H;
+
+    // hand-over slot fields
+    auto slot_ptr = [&](int i) { return scratch + (size_t)(i & 1) * SLOT; };
+    constexpr int oQ = 0, oK = D, oMK = 2 * D, oMQ = 3 * D, oLB = 4 * D, oLN = 5 * D, oB = 6 * D, oCK = 7 * D,
+                  oCQ = 7 * D + kMaxCap, oSC = 7 * D + 2 * kMaxCap, oRED = 7 * D + 2 * kMaxCap + 4;
+
+    if (warp == 2 * kGroupWarps) {
+        // ================= base-ring producer: needs only the slot of each unit ==================
+        RingPos pos;
+        bool dead = false;
+        long long issued = 0;
+        for (int it0 = 0; it0 < n_items; it0 += 32) {
+            int slot = -1;
+            if (it0 + lane < n_items) {
+                const int item = first + (it0 + lane) * stride;
+                slot = tk.slot_idx ? tk.slot_idx[item / H] : item / H;
+                if (slot >= st.num_slots) slot = -1;
+            }
+            const int cnt = min(32, n_items - it0);
+            for (int j = 0; j < cnt; ++j) {
+                const int s = __shfl_sync(0xffffffffu, slot, j);
+                if (s < 0 || lane != 0 || dead) continue;
+                const int h = (first + (it0 + j) * stride) % H;
+                const char *src = reinterpret_cast<const char *>(st.S_base + ((size_t)s * H + h) * D * D);
+                for (int c = 0; c < NCHUNK && !dead; ++c) {
+                    if (!bounded_wait(empty_base + 8u * pos.stage, pos.phase ^ 1u, abort_flag)) {
+                        dead = true;
+                        break;
+                    }
+                    const uint32_t fb = full_base + 8u * pos.stage;
+                    mbar_arrive_expect_tx(fb, kChunkBytes);
+                    bulk_copy_g2s(smem_addr(base_ring + (size_t)pos.stage * kChunkBytes), src + (size_t)c * kChunkBytes,
+                                  kChunkBytes, fb);
+                    pos.advance(NB);
+                    ++issued;
+                }
+            }
+        }
+        if (lane == 0 && dead) {  // wait out the copies still in flight before shared memory goes away
+            if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+            const int back = (int)min((long long)NB, issued);
+            for (int i = 0; i < back; ++i) {
+                int stg = pos.stage - 1 - i;
+                uint32_t ph = pos.phase;
+                if (stg < 0) {
+                    stg += NB;
+                    ph ^= 1u;
+                }
+                bounded_wait(full_base + 8u * stg, ph, abort_flag + 1);
+            }
+        }
+    } else if (warp == 2 * kGroupWarps + 1) {
+        // ================= aux-ring producer: metadata, live log entries, token vectors ==========
+        RingPos pos;
+        bool dead = false;
+        long long issued = 0;
+        const int io_vec = D * (int)sizeof(IO);
+        for (int it0 = 0; it0 < n_items; it0 += 32) {
+            int slot = -1, len = 0, flags = kMetaSkip;
+            float gs = 0.f, bt = 0.f;
+            if (it0 + lane < n_items) {
+                const int item = first + (it0 + lane) * stride;
+                slot = tk.slot_idx ? tk.slot_idx[item / H] : item / H;
+                if (slot >= st.num_slots) {
+                    if (st.status) atomicOr(st.status, DELTALOG_STATUS_BAD_SLOT);
+                    slot = -1;
+                }
+                if (slot >= 0) {
+                    len = st.log_len[(size_t)slot * H + item % H];
+                    flags = 0;
+                    if (len >= cap || len < 0) {
+                        if (st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
+                        flags = kMetaFull;
+                    }
+                    if (!kVecDecay) gs = tk.g[item];
+                    if (kDelta) bt = tk.beta[item];
+                }
+            }
+            const int cnt = min(32, n_items - it0);
+            for (int j = 0; j < cnt; ++j) {
+                const int s = __shfl_sync(0xffffffffu, slot, j);
+                const int L = __shfl_sync(0xffffffffu, len, j);
+                const int fl = __shfl_sync(0xffffffffu, flags, j);
+                const float gsj = __shfl_sync(0xffffffffu, gs, j);
+                const float btj = __shfl_sync(0xffffffffu, bt, j);
+                if (lane != 0 || dead) continue;
+                if (!bounded_wait(empty_aux + 8u * pos.stage, pos.phase ^ 1u, abort_flag)) {
+                    dead = true;
+                    continue;
+                }
+                unsigned char *stage = aux_ring + (size_t)pos.stage * lay.bytes;
+                *reinterpret_cast<int4 *>(stage + lay.meta) = make_int4(L, fl, __float_as_int(gsj), __float_as_int(btj));
+                *reinterpret_cast<int *>(stage + lay.meta + 16) = s;
+                const uint32_t fa = full_aux + 8u * pos.stage;
+                if (fl != 0) {
+                    mbar_arrive(fa);  // nothing to copy: the compute warps only read the flags
+                } else {
+                    const int item = first + (it0 + j) * stride;
+                    const size_t unit = (size_t)s * H + item % H;
+                    const int kb = L * D * (int)sizeof(IO), ub = L * D * (int)sizeof(UL);
+                    const int lb = kVecDecay ? L * D * 4 : align_up(L, 4) * 4;
+                    const uint32_t bytes = kb + ub + lb + 3 * io_vec + (kVecDecay ? D * 4 : 0) +
+                                           (OP == DELTALOG_RWKV6 ? D * 4 : 0);
+                    mbar_arrive_expect_tx(fa, bytes);
+                    const uint32_t sa = smem_addr(stage);
+                    bulk_copy_g2s(sa + lay.q, static_cast<const IO *>(tk.q) + (size_t)item * D, io_vec, fa);
+                    bulk_copy_g2s(sa + lay.k, static_cast<const IO *>(tk.k) + (size_t)item * D, io_vec, fa);
+                    if (kVecDecay) bulk_copy_g2s(sa + lay.g, tk.g + (size_t)item * D, D * 4, fa);
+                    if (L > 0) {
+                        bulk_copy_g2s(sa + lay.L, st.decay_log + unit * cap * DL, lb, fa);
+                        bulk_copy_g2s(sa + lay.K, static_cast<const IO *>(st.K_log) + unit * cap * D, kb, fa);
+                        bulk_copy_g2s(sa + lay.U, static_cast<const UL *>(st.U_log) + unit * cap * D, ub, fa);
+                    }
+                    bulk_copy_g2s(sa + lay.v, static_cast<const IO *>(tk.v) + (size_t)item * D, io_vec, fa);
+                    if (OP == DELTALOG_RWKV6) bulk_copy_g2s(sa + lay.bonus, tk.u_bonus + (size_t)(item % H) * D, D * 4, fa);
+                }
+                pos.advance(NA);
+                ++issued;
+            }
+        }
+        if (lane == 0 && dead) {
+            if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+            const int back = (int)min((long long)NA, issued);
+            for (int i = 0; i < back; ++i) {
+                int stg = pos.stage - 1 - i;
+                uint32_t ph = pos.phase;
+                if (stg < 0) {
+                    stg += NA;
+                    ph ^= 1u;
+                }
+                bounded_wait(full_aux + 8u * stg, ph, abort_flag + 1);
+            }
+        }
+    } else if (warp < kGroupWarps) {
+        // ================= stream group: the base pass, nothing else =============================
+        // Warps run independently of one another (no group barrier): each waits for the unit's
+        // multipliers, folds its rows of every chunk into its partial sums and hands them over.
+        const int c4 = tid % C4, rl = tid / C4;
+        RingPos bpos;
+        for (int it = 0; it < n_items; ++it) {
+            const uint32_t par = (uint32_t)(it >> 1) & 1u;
+            if (!bounded_wait(prep_done + 8u * (it & 1), par, abort_flag)) break;
+            float *sl = slot_ptr(it);
+            const int flags = __float_as_int(sl[oSC + 1]);
+            if (!(flags & kMetaSkip)) {
+                const float *mk_s = sl + oMK, *mq_s = sl + oMQ;
+                float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), aq = ak;
+                bool failed = false;
+#pragma unroll 1
+                for (int c = 0; c < NCHUNK; ++c) {
+                    if (!bounded_wait(full_base + 8u * bpos.stage, bpos.phase, abort_flag)) {
+                        failed = true;
+                        break;
+                    }
+                    if (!(flags & kMetaFull)) {
+                        const float4 *tile =
+                            reinterpret_cast<const float4 *>(base_ring + (size_t)bpos.stage * kChunkBytes);
+                        const int r0 = c * CH_ROWS + rl * PPC;  // this thread's four consecutive rows
+                        const float4 mq4 = *reinterpret_cast<const float4 *>(mq_s + r0);
+                        float4 mk4 = mq4;
+                        if (kDelta) mk4 = *reinterpret_cast<const float4 *>(mk_s + r0);
+                        const float4 x0 = tile[(rl * PPC + 0) * C4 + c4], x1 = tile[(rl * PPC + 1) * C4 + c4];
+                        const float4 x2 = tile[(rl * PPC + 2) * C4 + c4], x3 = tile[(rl * PPC + 3) * C4 + c4];
+                        if (kDelta) {
+                            ak = fma4(mk4.x, x0, ak);
+                            ak = fma4(mk4.y, x1, ak);
+                            ak = fma4(mk4.z, x2, ak);
+                            ak = fma4(mk4.w, x3, ak);
+                        }
+                        aq = fma4(mq4.x, x0, aq);
+                        aq = fma4(mq4.y, x1, aq);
+                        aq = fma4(mq4.z, x2, aq);
+                        aq = fma4(mq4.w, x3, aq);
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(empty_base + 8u * bpos.stage);
+                    bpos.advance(NB);
+                }
+                if (failed) break;
+                float4 *red4 = reinterpret_cast<float4 *>(sl + oRED);
+                if (kDelta) red4[(rl * 2 + 0) * C4 + c4] = ak;
+                red4[(rl * 2 + 1) * C4 + c4] = aq;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(stream_done + 8u * (it & 1));
+        }
+    } else {
+        // ================= scalar group: prep for unit i+1, epilogue of unit i ===================
+        const int gtid = tid - kPipeConsumers, gwarp = warp - kGroupWarps;
+        RingPos apos;       // aux stage of the next unit to prepare
+        bool alive = true;
+
+        // prep(j): cumulative decay, multipliers (-> stream group), replay coefficients, q.k
+        auto prep = [&](int j) -> bool {
+            const bool got = bounded_wait(full_aux + 8u * apos.stage, apos.phase, abort_flag);
+            if (consumers_any(!got)) return false;
+            const unsigned char *stage = aux_ring + (size_t)apos.stage * lay.bytes;
+            apos.advance(NA);
+            float *sl = slot_ptr(j);
+            const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
+            const int len = meta.x, flags = meta.y;
+            if (flags != 0) {
+                if (gtid == 0) {
+                    sl[oSC + 1] = __int_as_float(flags);
+                    mbar_arrive(prep_done + 8u * (j & 1));
+                }
+                return true;
+            }
+            const IO *q_a = reinterpret_cast<const IO *>(stage + lay.q);
+            const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
+            const IO *K_a = reinterpret_cast<const IO *>(stage + lay.K);
+            const float *L_a = reinterpret_cast<const float *>(stage + lay.L);
+            const float *g_a = reinterpret_cast<const float *>(stage + lay.g);
+            const float *bonus_a = reinterpret_cast<const float *>(stage + lay.bonus);
+            float *q_s = sl + oQ, *k_s = sl + oK, *lbar_s = sl + oLB;
+            if (gtid < D) {
+                const float qv = to_f32(q_a[gtid]);
+                const float kv = to_f32(k_a[gtid]);
+                const float lold = (len > 0) ? L_a[(len - 1) * DL + (kVecDecay ? gtid : 0)] : 0.f;
+                const float lnew = lold + (kVecDecay ? g_a[gtid] : __int_as_float(meta.z));
+                q_s[gtid] = qv;
+                k_s[gtid] = kv;
+                lbar_s[gtid] = kDelta ? lnew : lold;  // the decay level the readouts refer to
+                sl[oLN + gtid] = lnew;                // the level stored with the appended entry
+                const float e = expf(kDelta ? lnew : lold);
+                sl[oMK + gtid] = e * kv;
+                sl[oMQ + gtid] = e * qv;
+            }
+            if (gtid == 0) sl[oSC + 1] = __int_as_float(0);
+            consumers_sync();
+            if (gtid == 0) mbar_arrive(prep_done + 8u * (j & 1));  // the stream group may start on this unit
+
+            // key-side replay coefficients: each lane owns EPL consecutive key channels; a warp takes
+            // entries gwarp, gwarp+8, ... two at a time so that the shuffle reductions overlap
+            float qv[EPL], kv[EPL], lb[EPL];
+            load_vec<float, EPL>(q_s + lane * EPL, qv);
+            load_vec<float, EPL>(k_s + lane * EPL, kv);
+            if (kVecDecay) load_vec<float, EPL>(lbar_s + lane * EPL, lb);
+            for (int i0 = gwarp; i0 < len; i0 += 2 * kGroupWarps) {
+                const int i1 = i0 + kGroupWarps;
+                const bool two = i1 < len;
+                float dq0 = 0.f, dk0 = 0.f, dq1 = 0.f, dk1 = 0.f;
+                float ke[EPL], le[EPL];
+                load_vec<IO, EPL>(K_a + i0 * D + lane * EPL, ke);
+                if (kVecDecay) load_vec<float, EPL>(L_a + i0 * D + lane * EPL, le);
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) {
+                    const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
+                    dq0 = fmaf(qv[e], kij, dq0);
+                    if (kDelta) dk0 = fmaf(kv[e], kij, dk0);
+                }
+                if (two) {
+                    load_vec<IO, EPL>(K_a + i1 * D + lane * EPL, ke);
+                    if (kVecDecay) load_vec<float, EPL>(L_a + i1 * D + lane * EPL, le);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) {
+                        const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
+                        dq1 = fmaf(qv[e], kij, dq1);
+                        if (kDelta) dk1 = fmaf(kv[e], kij, dk1);
+                    }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    dq0 += __shfl_xor_sync(0xffffffffu, dq0, o);
+                    dq1 += __shfl_xor_sync(0xffffffffu, dq1, o);
+                    if (kDelta) {
+                        dk0 += __shfl_xor_sync(0xffffffffu, dk0, o);
+                        dk1 += __shfl_xor_sync(0xffffffffu, dk1, o);
+                    }
+                }
+                if (lane == 0) {
+                    const float w0 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i0]);
+                    sl[oCQ + i0] = w0 * dq0;
+                    if (kDelta) sl[oCK + i0] = w0 * dk0;
+                    if (two) {
+                        const float w1 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i1]);
+                        sl[oCQ + i1] = w1 * dq1;
+                        if (kDelta) sl[oCK + i1] = w1 * dk1;
+                    }
+                }
+            }
+            if (gwarp == kGroupWarps - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
+                float d = 0.f;
+                float bw[EPL];
+                if (!kDelta) load_vec<float, EPL>(bonus_a + lane * EPL, bw);
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) d = fmaf(kDelta ? qv[e] : qv[e] * bw[e], kv[e], d);
+                d = warp_sum(d);
+                if (lane == 0) sl[oSC] = d;
+            }
+            return true;
+        };
+
+        if (n_items > 0) alive = prep(0);
+        RingPos epos;  // aux stage of the unit whose epilogue runs
+        for (int it = 0; it < n_items && alive; ++it) {
+            if (it + 1 < n_items && !prep(it + 1)) {
+                alive = false;
+                break;
+            }
+            // ---- epilogue of unit `it` ----------------------------------------------------------
+            const uint32_t par = (uint32_t)(it >> 1) & 1u;
+            const bool got = bounded_wait(stream_done + 8u * (it & 1), par, abort_flag);
+            if (consumers_any(!got)) {  // also orders this unit's coefficient writes before their use
+                alive = false;
+                break;
+            }
+            const unsigned char *stage = aux_ring + (size_t)epos.stage * lay.bytes;
+            const uint32_t ea = empty_aux + 8u * epos.stage;
+            epos.advance(NA);
+            const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
+            const int len = meta.x, flags = meta.y;
+            if (flags == 0) {
+                const int slot = *reinterpret_cast<const int *>(stage + lay.meta + 16);
+                const int item = first + it * stride;
+                const size_t unit = (size_t)slot * H + item % H;
+                const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
+                const IO *v_a = reinterpret_cast<const IO *>(stage + lay.v);
+                const UL *U_a = reinterpret_cast<const UL *>(stage + lay.U);
+                float *sl = slot_ptr(it);
+                const float *red_s = sl + oRED;
+                float *b_s = sl + oB;
+                const int which = gtid / D, c = gtid % D;  // which: 0 -> y_k half, 1 -> y_q half
+                const bool active = kDelta ? (gtid < 2 * D) : (gtid < D);
+                const int sel = kDelta ? which : 1;
+                float y = 0.f;
+                if (active) {
+#pragma unroll
+                    for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+                    const float *coef = sl + (sel ? oCQ : oCK);
+                    float y1 = 0.f;
+                    int i = 0;
+#pragma unroll 4
+                    for (; i + 1 < len; i += 2) {
+                        y = fmaf(coef[i], to_f32(U_a[i * D + c]), y);
+                        y1 = fmaf(coef[i + 1], to_f32(U_a[(i + 1) * D + c]), y1);
+                    }
+                    if (i < len) y = fmaf(coef[i], to_f32(U_a[i * D + c]), y);
+                    y += y1;
+                }
+                UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
+                IO *og = static_cast<IO *>(tk.out) + (size_t)item * D;
+                if (kDelta) {
+                    if (gtid < D) {
+                        const float bval = __int_as_float(meta.w) * (to_f32(v_a[c]) - y);
+                        b_s[c] = bval;
+                        Uout[c] = from_f32<UL>(bval);
+                    }
+                    consumers_sync();
+                    if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(sl[oSC], b_s[c], y));
+                } else if (active) {
+                    const IO v_raw = v_a[c];
+                    og[c] = from_f32<IO>(fmaf(sl[oSC], to_f32(v_raw), y));
+                    Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+                }
+                if (gtid < D) {
+                    (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[gtid] = k_a[gtid];
+                    if (kVecDecay) st.decay_log[(unit * cap + len) * DL + gtid] = sl[oLN + gtid];
+                }
+                if (gtid == 0) {
+                    if (!kVecDecay) st.decay_log[unit * cap + len] = sl[oLN];
+                    st.log_len[unit] = len + 1;
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ea);  // this warp is done with the unit's aux stage
+        }
+        if (!alive && gtid == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+    }
+}
+
+}  // namespace deltalog

@@ -4,7 +4,10 @@
 #include <cstdint>
 #include <type_traits>
 
+#include <cstdlib>
+
 #include "decode_kernel.cuh"
+#include "decode_pipelined.cuh"
 #include "eager_kernel.cuh"
 #include "merge_kernel.cuh"
 
@@ -77,13 +80,76 @@ int ensure_smem(K kernel, size_t bytes) {
     return DELTALOG_OK;
 }
 
+// Device facts needed to size the persistent kernel, queried once per device.
+struct DeviceInfo {
+    int sms = 0;
+    int smem_per_sm = 0;
+    int smem_optin = 0;
+};
+const DeviceInfo &device_info() {
+    static DeviceInfo info[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    DeviceInfo &d = info[dev & 63];
+    if (d.sms == 0) {
+        cudaDeviceGetAttribute(&d.smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, dev);
+        cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev);
+    }
+    return d;
+}
+
+// Tuning knobs (environment, read once): DELTALOG_DECODE_IMPL = 0 auto | 1 one-CTA-per-unit | 2 pipelined;
+// DELTALOG_CTAS_PER_SM, DELTALOG_BASE_STAGES, DELTALOG_AUX_STAGES override the pipelined kernel's shape.
+int env_int(const char *name, int dflt) {
+    const char *v = std::getenv(name);
+    return v ? std::atoi(v) : dflt;
+}
+
 template <int OP, int D, typename IO>
 int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
     using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
+    static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
+    static const int env_base = env_int("DELTALOG_BASE_STAGES", 0);
+    static const int env_aux = env_int("DELTALOG_AUX_STAGES", 0);
+    const DeviceInfo &dev = device_info();
+    const int total = tk.B * st.H;
+
+    // The pipelined kernel moves the scalar decay snapshots with 16-byte bulk copies, which needs
+    // every unit's snapshot row to start on a 16-byte boundary: cap % 4 == 0 for GDN.
+    bool pipelined = impl != 1 && dev.sms > 0 && (OP != DELTALOG_GDN || st.cap % 4 == 0);
+    PipeCfg cfg{0, 0};
+    int ctas = env_ctas > 0 ? env_ctas : 1;
+    if (pipelined) {
+        const int aux = AuxLayout<OP, D, IO, UL>(st.cap).bytes;
+        const int fixed = kPipeBarrierBytes + pipe_scratch_bytes<D>();
+        const int want_base = env_base > 0 ? env_base : 8;  // 128 KiB in flight per SM saturates HBM
+        for (; ctas >= 1; --ctas) {
+            int budget = dev.smem_per_sm / ctas - 1024;
+            if (budget > dev.smem_optin) budget = dev.smem_optin;
+            // aux stages: two are held by the scalar group (unit i and i+1), the rest is prefetch
+            for (cfg.n_aux = env_aux > 0 ? env_aux : 4; cfg.n_aux >= 2; --cfg.n_aux) {
+                cfg.n_base = (budget - fixed - cfg.n_aux * aux) / kChunkBytes;
+                if (cfg.n_base >= want_base || (cfg.n_aux == 2 && cfg.n_base >= 2)) break;
+            }
+            if (cfg.n_aux >= 2) break;
+        }
+        if (ctas < 1) pipelined = false;
+        if (cfg.n_base > want_base) cfg.n_base = want_base;
+    }
+    if (pipelined) {
+        auto kernel = decode_pipelined_kernel<OP, D, IO, UL>;
+        const int smem = pipe_smem_bytes<OP, D, IO, UL>(st.cap, cfg);
+        if (int rc = ensure_smem(kernel, smem)) return rc;
+        const int grid = total < dev.sms * ctas ? total : dev.sms * ctas;
+        kernel<<<grid, kPipeThreads, smem, stream>>>(st, tk, cfg);
+        return finish_launch();
+    }
     auto kernel = decode_append_kernel<OP, D, IO, UL>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<tk.B * st.H, kThreads, smem, stream>>>(st, tk);
+    kernel<<<total, kThreads, smem, stream>>>(st, tk);
     return finish_launch();
 }
 
