@@ -1,28 +1,30 @@
-// Persistent, warp-specialised decode + append kernel.
+// Persistent, warp-specialised decode + append kernel (head size 128).
 //
 // Same arithmetic as decode_append_kernel (Algorithm 1, append branch; Eq. 4 and Eq. 6), different
 // schedule.  One CTA stays resident per SM and walks over its share of the (batch row, head) units.
-// Four roles run concurrently and hand work to one another through mbarriers:
+// Five roles run concurrently and hand work to one another through mbarriers:
 //
-//   base producer (1 warp)  bulk asynchronous copies (cp.async.bulk) of 16 KiB chunks of the fp32
-//                           base tile (d=128: 4 chunks per unit, d=64: 1) into the base ring;
-//   aux producer  (1 warp)  per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
-//                           token vectors q, k, v (and g, bonus where they are vectors) and a small
-//                           metadata record (len, flags, scalar gate, beta) into the aux ring;
-//   stream group  (8 warps) the base pass only: the two mat-vecs S_base^T (e^lbar . k) and
-//                           S_base^T (e^lbar . q) from each chunk the moment it lands, releasing the
-//                           chunk at once, so the HBM stream never waits for a unit's epilogue;
-//   scalar group  (8 warps) everything that does not touch the base: for unit i+1 the cumulative
-//                           decay, the decayed multipliers and the key-side replay coefficients
-//                           (the paper's ReplayPrep, here a pipeline stage instead of a launch); for
-//                           unit i the cross-warp reduction, the value-side replay, b, the output and
-//                           the append.
+//   base producer  (1 warp)  bulk asynchronous copies (cp.async.bulk, completion counted on
+//                            mbarriers) of 16 KiB chunks of the fp32 base tile -- the only large
+//                            read -- into the base ring, the four chunks of a unit issued by four
+//                            lanes in lockstep; a chunk's stage is refilled the moment it has been
+//                            consumed, so the HBM stream never waits for a unit's epilogue;
+//   aux producer   (1 warp)  per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
+//                            token vectors q, k, v (and g, bonus where they are vectors) and a small
+//                            metadata record written by the producer (len, flags, scalar gate, beta)
+//                            into the aux ring;
+//   stream group   (8 warps) the base pass only: the two mat-vecs S_base^T (e^lbar . k) and
+//                            S_base^T (e^lbar . q) from each chunk as it lands;
+//   prep group     (4 warps) for unit i+1: cumulative decay, decayed multipliers (handed to the
+//                            stream group) and the key-side replay coefficients -- the paper's
+//                            ReplayPrep, here a pipeline stage instead of a launch;
+//   epilogue group (4 warps) for unit i, once the stream group is through it: cross-warp
+//                            reduction, value-side replay, b, the output and the append.
 //
-// No compute warp ever issues a global load; what the scalar group writes (out, the appended entry
-// and the new length) is fire-and-forget.  Every wait on an mbarrier is bounded in time: when it
-// gives up it raises the CTA's abort flag, ORs DELTALOG_STATUS_TIMEOUT into the status word, and all
-// roles leave their loops; the producers then wait (bounded again) for the copies they still have
-// in flight before the CTA exits.
+// No compute warp ever issues a global load; what the epilogue group writes (out, the appended
+// entry and the new length) is fire-and-forget.  Every wait on an mbarrier is bounded in time:
+// when it gives up it raises the CTA's abort flag, ORs DELTALOG_STATUS_TIMEOUT into the status
+// word, and all roles leave their loops.
 #pragma once
 
 #include "common.cuh"
@@ -59,11 +61,11 @@ struct AuxLayout {
 };
 
 // Hand-over buffer between the roles, two slots (unit i and unit i+1 are in flight together).
-// Per slot (floats): q, k, mul_k, mul_q, lbar, lbar', b [7*D], ck, cq [2*64], scalars [4]: q.k and the
+// Per slot (floats): q, k, mul_k, mul_q, lbar, lbar' [6*D], ck, cq [2*64], scalars [4]: q.k and the
 // unit's flags; then the stream group's partial sums [RL][2][D].
 template <int D>
 __host__ __device__ constexpr int pipe_slot_floats() {
-    return 7 * D + 2 * kMaxCap + 4 + 2 * D * (kPipeConsumers / (D / 4));
+    return 6 * D + 2 * kMaxCap + 4 + 2 * D * (kPipeConsumers / (D / 4));
 }
 template <int D>
 __host__ __device__ constexpr int pipe_scratch_bytes() {
@@ -143,6 +145,18 @@ __device__ __forceinline__ void consumers_sync() {
     asm volatile("bar.sync 1, %0;\n" ::"n"(kPipeConsumers) : "memory");
 }
 
+// The same for one of the two 128-thread scalar groups (named barrier `id`).
+__device__ __forceinline__ bool group_any(bool pred, int id) {
+    uint32_t res;
+    asm volatile(
+        "{\n .reg .pred p, q;\n setp.ne.u32 q, %1, 0;\n bar.red.or.pred p, %2, 128, q;\n selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(res)
+        : "r"((uint32_t)pred), "r"(id)
+        : "memory");
+    return res != 0;
+}
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;\n" ::"r"(id) : "memory"); }
+
 struct RingPos {  // position in a ring of n stages: stage index and phase parity
     int stage = 0;
     uint32_t phase = 0;
@@ -182,7 +196,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     const uint32_t full_base = smem_addr(bars), empty_base = full_base + 8u * NB;
     const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * NA;
     const uint32_t prep_done = empty_aux + 8u * NA;   // [2] scalar group -> stream group: multipliers ready
-    const uint32_t stream_done = prep_done + 16u;     // [2] stream group -> scalar group: partial sums ready
+    const uint32_t stream_done = prep_done + 16u;     // [2] stream group -> epilogue group: partial sums ready
+    const uint32_t coef_done = stream_done + 16u;     // [2] prep group -> epilogue group: coefficients ready
+    const uint32_t slot_free = coef_done + 16u;       // [2] epilogue group -> prep group: hand-over slot reusable
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -197,6 +213,8 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         for (int i = 0; i < 2; ++i) {
             mbar_init(prep_done + 8u * i, 1);
             mbar_init(stream_done + 8u * i, kGroupWarps);
+            mbar_init(coef_done + 8u * i, kGroupWarps / 2);
+            mbar_init(slot_free + 8u * i, kGroupWarps / 2);
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;  // separate flag for the drain waits after an abort
@@ -212,14 +230,14 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
 
     // hand-over slot fields
     auto slot_ptr = [&](int i) { return scratch + (size_t)(i & 1) * SLOT; };
-    constexpr int oQ = 0, oK = D, oMK = 2 * D, oMQ = 3 * D, oLB = 4 * D, oLN = 5 * D, oB = 6 * D, oCK = 7 * D,
-                  oCQ = 7 * D + kMaxCap, oSC = 7 * D + 2 * kMaxCap, oRED = 7 * D + 2 * kMaxCap + 4;
+    constexpr int oQ = 0, oK = D, oMK = 2 * D, oMQ = 3 * D, oLB = 4 * D, oLN = 5 * D, oCK = 6 * D,
+                  oCQ = 6 * D + kMaxCap, oSC = 6 * D + 2 * kMaxCap, oRED = 6 * D + 2 * kMaxCap + 4;
 
     if (warp == 2 * kGroupWarps) {
         // ================= base-ring producer: needs only the slot of each unit ==================
-        RingPos pos;
+        // The NCHUNK chunks of a unit are issued by NCHUNK lanes in lockstep (lane c handles chunk c).
         bool dead = false;
-        long long issued = 0;
+        int m = 0;  // chunks queued so far (warp-uniform)
         for (int it0 = 0; it0 < n_items; it0 += 32) {
             int slot = -1;
             if (it0 + lane < n_items) {
@@ -230,36 +248,27 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             const int cnt = min(32, n_items - it0);
             for (int j = 0; j < cnt; ++j) {
                 const int s = __shfl_sync(0xffffffffu, slot, j);
-                if (s < 0 || lane != 0 || dead) continue;
+                if (s < 0) continue;
                 const int h = (first + (it0 + j) * stride) % H;
                 const char *src = reinterpret_cast<const char *>(st.S_base + ((size_t)s * H + h) * D * D);
-                for (int c = 0; c < NCHUNK && !dead; ++c) {
-                    if (!bounded_wait(empty_base + 8u * pos.stage, pos.phase ^ 1u, abort_flag)) {
+                if (lane < NCHUNK && !dead) {
+                    const int mm = m + lane;
+                    const int stage = mm % NB;
+                    const uint32_t phase = (uint32_t)(mm / NB) & 1u;
+                    if (!bounded_wait(empty_base + 8u * stage, phase ^ 1u, abort_flag)) {
                         dead = true;
-                        break;
+                    } else {
+                        const uint32_t fb = full_base + 8u * stage;
+                        mbar_arrive_expect_tx(fb, kChunkBytes);
+                        bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * kChunkBytes), src + (size_t)lane * kChunkBytes,
+                                      kChunkBytes, fb);
                     }
-                    const uint32_t fb = full_base + 8u * pos.stage;
-                    mbar_arrive_expect_tx(fb, kChunkBytes);
-                    bulk_copy_g2s(smem_addr(base_ring + (size_t)pos.stage * kChunkBytes), src + (size_t)c * kChunkBytes,
-                                  kChunkBytes, fb);
-                    pos.advance(NB);
-                    ++issued;
                 }
+                __syncwarp();
+                m += NCHUNK;
             }
         }
-        if (lane == 0 && dead) {  // wait out the copies still in flight before shared memory goes away
-            if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
-            const int back = (int)min((long long)NB, issued);
-            for (int i = 0; i < back; ++i) {
-                int stg = pos.stage - 1 - i;
-                uint32_t ph = pos.phase;
-                if (stg < 0) {
-                    stg += NB;
-                    ph ^= 1u;
-                }
-                bounded_wait(full_base + 8u * stg, ph, abort_flag + 1);
-            }
-        }
+        if (__any_sync(0xffffffffu, dead) && lane == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
     } else if (warp == 2 * kGroupWarps + 1) {
         // ================= aux-ring producer: metadata, live log entries, token vectors ==========
         RingPos pos;
@@ -396,185 +405,182 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             if (lane == 0) mbar_arrive(stream_done + 8u * (it & 1));
         }
     } else {
-        // ================= scalar group: prep for unit i+1, epilogue of unit i ===================
-        const int gtid = tid - kPipeConsumers, gwarp = warp - kGroupWarps;
-        RingPos apos;       // aux stage of the next unit to prepare
+        // ================= scalar groups ==========================================================
+        // Two groups of four warps split the non-streaming work of every unit by function, so that
+        // the preparation of unit i+1 runs beside the epilogue of unit i:
+        //   prep group      cumulative decay, decayed multipliers (-> stream group), key-side replay
+        //                   coefficients and q.k (-> epilogue group);
+        //   epilogue group  cross-warp reduction, value-side replay, b, output, append.
+        constexpr int kHalf = kGroupWarps / 2;
+        const bool is_prep = warp < kGroupWarps + kHalf;
+        const int gtid = tid - kPipeConsumers - (is_prep ? 0 : 32 * kHalf), gwarp = gtid >> 5;
         bool alive = true;
+        if (is_prep) {
+            for (int j = 0; j < n_items; ++j) {
+                const int stg = j % NA;
+                bool got = bounded_wait(full_aux + 8u * stg, (uint32_t)(j / NA) & 1u, abort_flag);
+                got = got && bounded_wait(slot_free + 8u * (j & 1), ((uint32_t)(j >> 1) & 1u) ^ 1u, abort_flag);
+                if (group_any(!got, 1)) {
+                    alive = false;
+                    break;
+                }
+                const unsigned char *stage = aux_ring + (size_t)stg * lay.bytes;
+                float *sl = slot_ptr(j);
+                const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
+                const int len = meta.x, flags = meta.y;
+                if (flags == 0) {
+                    const IO *q_a = reinterpret_cast<const IO *>(stage + lay.q);
+                    const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
+                    const IO *K_a = reinterpret_cast<const IO *>(stage + lay.K);
+                    const float *L_a = reinterpret_cast<const float *>(stage + lay.L);
+                    const float *g_a = reinterpret_cast<const float *>(stage + lay.g);
+                    const float *bonus_a = reinterpret_cast<const float *>(stage + lay.bonus);
+                    float *q_s = sl + oQ, *k_s = sl + oK, *lbar_s = sl + oLB;
+                    if (gtid < D) {
+                        const float qv = to_f32(q_a[gtid]);
+                        const float kv = to_f32(k_a[gtid]);
+                        const float lold = (len > 0) ? L_a[(len - 1) * DL + (kVecDecay ? gtid : 0)] : 0.f;
+                        const float lnew = lold + (kVecDecay ? g_a[gtid] : __int_as_float(meta.z));
+                        q_s[gtid] = qv;
+                        k_s[gtid] = kv;
+                        lbar_s[gtid] = kDelta ? lnew : lold;  // the decay level the readouts refer to
+                        sl[oLN + gtid] = lnew;                // the level stored with the appended entry
+                        const float e = expf(kDelta ? lnew : lold);
+                        sl[oMK + gtid] = e * kv;
+                        sl[oMQ + gtid] = e * qv;
+                    }
+                    if (gtid == 0) sl[oSC + 1] = __int_as_float(0);
+                    group_sync(1);
+                    if (gtid == 0) mbar_arrive(prep_done + 8u * (j & 1));  // the stream group may start on this unit
 
-        // prep(j): cumulative decay, multipliers (-> stream group), replay coefficients, q.k
-        auto prep = [&](int j) -> bool {
-            const bool got = bounded_wait(full_aux + 8u * apos.stage, apos.phase, abort_flag);
-            if (consumers_any(!got)) return false;
-            const unsigned char *stage = aux_ring + (size_t)apos.stage * lay.bytes;
-            apos.advance(NA);
-            float *sl = slot_ptr(j);
-            const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
-            const int len = meta.x, flags = meta.y;
-            if (flags != 0) {
-                if (gtid == 0) {
+                    // key-side replay coefficients: each lane owns EPL consecutive key channels; a warp
+                    // takes entries gwarp, gwarp+4, ... two at a time so that their reductions overlap
+                    float qv[EPL], kv[EPL], lb[EPL];
+                    load_vec<float, EPL>(q_s + lane * EPL, qv);
+                    load_vec<float, EPL>(k_s + lane * EPL, kv);
+                    if (kVecDecay) load_vec<float, EPL>(lbar_s + lane * EPL, lb);
+                    for (int i0 = gwarp; i0 < len; i0 += 2 * kHalf) {
+                        const int i1 = i0 + kHalf;
+                        const bool two = i1 < len;
+                        float dq0 = 0.f, dk0 = 0.f, dq1 = 0.f, dk1 = 0.f;
+                        float ke[EPL], le[EPL];
+                        load_vec<IO, EPL>(K_a + i0 * D + lane * EPL, ke);
+                        if (kVecDecay) load_vec<float, EPL>(L_a + i0 * D + lane * EPL, le);
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) {
+                            const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
+                            dq0 = fmaf(qv[e], kij, dq0);
+                            if (kDelta) dk0 = fmaf(kv[e], kij, dk0);
+                        }
+                        if (two) {
+                            load_vec<IO, EPL>(K_a + i1 * D + lane * EPL, ke);
+                            if (kVecDecay) load_vec<float, EPL>(L_a + i1 * D + lane * EPL, le);
+#pragma unroll
+                            for (int e = 0; e < EPL; ++e) {
+                                const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
+                                dq1 = fmaf(qv[e], kij, dq1);
+                                if (kDelta) dk1 = fmaf(kv[e], kij, dk1);
+                            }
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            dq0 += __shfl_xor_sync(0xffffffffu, dq0, o);
+                            dq1 += __shfl_xor_sync(0xffffffffu, dq1, o);
+                            if (kDelta) {
+                                dk0 += __shfl_xor_sync(0xffffffffu, dk0, o);
+                                dk1 += __shfl_xor_sync(0xffffffffu, dk1, o);
+                            }
+                        }
+                        if (lane == 0) {
+                            const float w0 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i0]);
+                            sl[oCQ + i0] = w0 * dq0;
+                            if (kDelta) sl[oCK + i0] = w0 * dk0;
+                            if (two) {
+                                const float w1 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i1]);
+                                sl[oCQ + i1] = w1 * dq1;
+                                if (kDelta) sl[oCK + i1] = w1 * dk1;
+                            }
+                        }
+                    }
+                    if (gwarp == kHalf - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
+                        float d = 0.f;
+                        float bw[EPL];
+                        if (!kDelta) load_vec<float, EPL>(bonus_a + lane * EPL, bw);
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) d = fmaf(kDelta ? qv[e] : qv[e] * bw[e], kv[e], d);
+                        d = warp_sum(d);
+                        if (lane == 0) sl[oSC] = d;
+                    }
+                } else if (gtid == 0) {
                     sl[oSC + 1] = __int_as_float(flags);
                     mbar_arrive(prep_done + 8u * (j & 1));
                 }
-                return true;
-            }
-            const IO *q_a = reinterpret_cast<const IO *>(stage + lay.q);
-            const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
-            const IO *K_a = reinterpret_cast<const IO *>(stage + lay.K);
-            const float *L_a = reinterpret_cast<const float *>(stage + lay.L);
-            const float *g_a = reinterpret_cast<const float *>(stage + lay.g);
-            const float *bonus_a = reinterpret_cast<const float *>(stage + lay.bonus);
-            float *q_s = sl + oQ, *k_s = sl + oK, *lbar_s = sl + oLB;
-            if (gtid < D) {
-                const float qv = to_f32(q_a[gtid]);
-                const float kv = to_f32(k_a[gtid]);
-                const float lold = (len > 0) ? L_a[(len - 1) * DL + (kVecDecay ? gtid : 0)] : 0.f;
-                const float lnew = lold + (kVecDecay ? g_a[gtid] : __int_as_float(meta.z));
-                q_s[gtid] = qv;
-                k_s[gtid] = kv;
-                lbar_s[gtid] = kDelta ? lnew : lold;  // the decay level the readouts refer to
-                sl[oLN + gtid] = lnew;                // the level stored with the appended entry
-                const float e = expf(kDelta ? lnew : lold);
-                sl[oMK + gtid] = e * kv;
-                sl[oMQ + gtid] = e * qv;
-            }
-            if (gtid == 0) sl[oSC + 1] = __int_as_float(0);
-            consumers_sync();
-            if (gtid == 0) mbar_arrive(prep_done + 8u * (j & 1));  // the stream group may start on this unit
-
-            // key-side replay coefficients: each lane owns EPL consecutive key channels; a warp takes
-            // entries gwarp, gwarp+8, ... two at a time so that the shuffle reductions overlap
-            float qv[EPL], kv[EPL], lb[EPL];
-            load_vec<float, EPL>(q_s + lane * EPL, qv);
-            load_vec<float, EPL>(k_s + lane * EPL, kv);
-            if (kVecDecay) load_vec<float, EPL>(lbar_s + lane * EPL, lb);
-            for (int i0 = gwarp; i0 < len; i0 += 2 * kGroupWarps) {
-                const int i1 = i0 + kGroupWarps;
-                const bool two = i1 < len;
-                float dq0 = 0.f, dk0 = 0.f, dq1 = 0.f, dk1 = 0.f;
-                float ke[EPL], le[EPL];
-                load_vec<IO, EPL>(K_a + i0 * D + lane * EPL, ke);
-                if (kVecDecay) load_vec<float, EPL>(L_a + i0 * D + lane * EPL, le);
-#pragma unroll
-                for (int e = 0; e < EPL; ++e) {
-                    const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
-                    dq0 = fmaf(qv[e], kij, dq0);
-                    if (kDelta) dk0 = fmaf(kv[e], kij, dk0);
-                }
-                if (two) {
-                    load_vec<IO, EPL>(K_a + i1 * D + lane * EPL, ke);
-                    if (kVecDecay) load_vec<float, EPL>(L_a + i1 * D + lane * EPL, le);
-#pragma unroll
-                    for (int e = 0; e < EPL; ++e) {
-                        const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
-                        dq1 = fmaf(qv[e], kij, dq1);
-                        if (kDelta) dk1 = fmaf(kv[e], kij, dk1);
-                    }
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    dq0 += __shfl_xor_sync(0xffffffffu, dq0, o);
-                    dq1 += __shfl_xor_sync(0xffffffffu, dq1, o);
-                    if (kDelta) {
-                        dk0 += __shfl_xor_sync(0xffffffffu, dk0, o);
-                        dk1 += __shfl_xor_sync(0xffffffffu, dk1, o);
-                    }
-                }
+                __syncwarp();
                 if (lane == 0) {
-                    const float w0 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i0]);
-                    sl[oCQ + i0] = w0 * dq0;
-                    if (kDelta) sl[oCK + i0] = w0 * dk0;
-                    if (two) {
-                        const float w1 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i1]);
-                        sl[oCQ + i1] = w1 * dq1;
-                        if (kDelta) sl[oCK + i1] = w1 * dk1;
-                    }
+                    mbar_arrive(coef_done + 8u * (j & 1));  // this warp's coefficients are in the slot
+                    mbar_arrive(empty_aux + 8u * stg);      // ... and it is done with the unit's aux stage
                 }
             }
-            if (gwarp == kGroupWarps - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
-                float d = 0.f;
-                float bw[EPL];
-                if (!kDelta) load_vec<float, EPL>(bonus_a + lane * EPL, bw);
+        } else {
+            for (int it = 0; it < n_items; ++it) {
+                const int stg = it % NA;
+                const uint32_t par = (uint32_t)(it >> 1) & 1u;
+                bool got = bounded_wait(stream_done + 8u * (it & 1), par, abort_flag);
+                got = got && bounded_wait(coef_done + 8u * (it & 1), par, abort_flag);
+                got = got && bounded_wait(full_aux + 8u * stg, (uint32_t)(it / NA) & 1u, abort_flag);
+                if (group_any(!got, 2)) {
+                    alive = false;
+                    break;
+                }
+                const unsigned char *stage = aux_ring + (size_t)stg * lay.bytes;
+                const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
+                const int len = meta.x, flags = meta.y;
+                if (flags == 0 && gtid < D) {  // this thread owns output column c: both readouts, b, the output
+                    const int slot = *reinterpret_cast<const int *>(stage + lay.meta + 16);
+                    const int item = first + it * stride;
+                    const size_t unit = (size_t)slot * H + item % H;
+                    const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
+                    const IO *v_a = reinterpret_cast<const IO *>(stage + lay.v);
+                    const UL *U_a = reinterpret_cast<const UL *>(stage + lay.U);
+                    const float *sl = slot_ptr(it);
+                    const float *red_s = sl + oRED;
+                    const int c = gtid;
+                    float yk = 0.f, yq = 0.f;
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) d = fmaf(kDelta ? qv[e] : qv[e] * bw[e], kv[e], d);
-                d = warp_sum(d);
-                if (lane == 0) sl[oSC] = d;
-            }
-            return true;
-        };
-
-        if (n_items > 0) alive = prep(0);
-        RingPos epos;  // aux stage of the unit whose epilogue runs
-        for (int it = 0; it < n_items && alive; ++it) {
-            if (it + 1 < n_items && !prep(it + 1)) {
-                alive = false;
-                break;
-            }
-            // ---- epilogue of unit `it` ----------------------------------------------------------
-            const uint32_t par = (uint32_t)(it >> 1) & 1u;
-            const bool got = bounded_wait(stream_done + 8u * (it & 1), par, abort_flag);
-            if (consumers_any(!got)) {  // also orders this unit's coefficient writes before their use
-                alive = false;
-                break;
-            }
-            const unsigned char *stage = aux_ring + (size_t)epos.stage * lay.bytes;
-            const uint32_t ea = empty_aux + 8u * epos.stage;
-            epos.advance(NA);
-            const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
-            const int len = meta.x, flags = meta.y;
-            if (flags == 0) {
-                const int slot = *reinterpret_cast<const int *>(stage + lay.meta + 16);
-                const int item = first + it * stride;
-                const size_t unit = (size_t)slot * H + item % H;
-                const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
-                const IO *v_a = reinterpret_cast<const IO *>(stage + lay.v);
-                const UL *U_a = reinterpret_cast<const UL *>(stage + lay.U);
-                float *sl = slot_ptr(it);
-                const float *red_s = sl + oRED;
-                float *b_s = sl + oB;
-                const int which = gtid / D, c = gtid % D;  // which: 0 -> y_k half, 1 -> y_q half
-                const bool active = kDelta ? (gtid < 2 * D) : (gtid < D);
-                const int sel = kDelta ? which : 1;
-                float y = 0.f;
-                if (active) {
-#pragma unroll
-                    for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
-                    const float *coef = sl + (sel ? oCQ : oCK);
-                    float y1 = 0.f;
-                    int i = 0;
+                    for (int r = 0; r < RL; ++r) {
+                        if (kDelta) yk += red_s[(r * 2 + 0) * D + c];
+                        yq += red_s[(r * 2 + 1) * D + c];
+                    }
 #pragma unroll 4
-                    for (; i + 1 < len; i += 2) {
-                        y = fmaf(coef[i], to_f32(U_a[i * D + c]), y);
-                        y1 = fmaf(coef[i + 1], to_f32(U_a[(i + 1) * D + c]), y1);
+                    for (int i = 0; i < len; ++i) {
+                        const float u = to_f32(U_a[i * D + c]);
+                        if (kDelta) yk = fmaf(sl[oCK + i], u, yk);
+                        yq = fmaf(sl[oCQ + i], u, yq);
                     }
-                    if (i < len) y = fmaf(coef[i], to_f32(U_a[i * D + c]), y);
-                    y += y1;
-                }
-                UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
-                IO *og = static_cast<IO *>(tk.out) + (size_t)item * D;
-                if (kDelta) {
-                    if (gtid < D) {
-                        const float bval = __int_as_float(meta.w) * (to_f32(v_a[c]) - y);
-                        b_s[c] = bval;
-                        Uout[c] = from_f32<UL>(bval);
-                    }
-                    consumers_sync();
-                    if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(sl[oSC], b_s[c], y));
-                } else if (active) {
                     const IO v_raw = v_a[c];
-                    og[c] = from_f32<IO>(fmaf(sl[oSC], to_f32(v_raw), y));
-                    Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+                    UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
+                    IO *og = static_cast<IO *>(tk.out) + (size_t)item * D;
+                    if (kDelta) {
+                        const float bval = __int_as_float(meta.w) * (to_f32(v_raw) - yk);
+                        Uout[c] = from_f32<UL>(bval);
+                        og[c] = from_f32<IO>(st.scale * fmaf(sl[oSC], bval, yq));
+                    } else {
+                        Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+                        og[c] = from_f32<IO>(fmaf(sl[oSC], to_f32(v_raw), yq));
+                    }
+                    (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[c] = k_a[c];
+                    if (kVecDecay) st.decay_log[(unit * cap + len) * DL + c] = sl[oLN + c];
+                    if (c == 0) {
+                        if (!kVecDecay) st.decay_log[unit * cap + len] = sl[oLN];
+                        st.log_len[unit] = len + 1;
+                    }
                 }
-                if (gtid < D) {
-                    (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[gtid] = k_a[gtid];
-                    if (kVecDecay) st.decay_log[(unit * cap + len) * DL + gtid] = sl[oLN + gtid];
-                }
-                if (gtid == 0) {
-                    if (!kVecDecay) st.decay_log[unit * cap + len] = sl[oLN];
-                    st.log_len[unit] = len + 1;
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(slot_free + 8u * (it & 1));  // the prep group may reuse the hand-over slot
+                    mbar_arrive(empty_aux + 8u * stg);       // this warp is done with the unit's aux stage
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(ea);  // this warp is done with the unit's aux stage
         }
         if (!alive && gtid == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
     }

@@ -118,7 +118,9 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
 
     // The pipelined kernel moves the scalar decay snapshots with 16-byte bulk copies, which needs
     // every unit's snapshot row to start on a 16-byte boundary: cap % 4 == 0 for GDN.
-    bool pipelined = impl != 1 && dev.sms > 0 && (OP != DELTALOG_GDN || st.cap % 4 == 0);
+    // Head size 64: a unit is a single 16 KiB chunk and the per-unit hand-overs of the pipeline cost
+    // more than they hide, so the one-CTA-per-unit kernel is the faster one there (measured).
+    bool pipelined = impl != 1 && dev.sms > 0 && (OP != DELTALOG_GDN || st.cap % 4 == 0) && (D == 128 || impl == 2);
     PipeCfg cfg{0, 0};
     int ctas = env_ctas > 0 ? env_ctas : 1;
     if (pipelined) {
