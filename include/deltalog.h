@@ -50,7 +50,8 @@ enum {
     DELTALOG_ERR_INVALID_ARG = 1,       /* NULL where a pointer is required, B < 0, bad enum, misaligned pointer */
     DELTALOG_ERR_UNSUPPORTED_SHAPE = 2, /* d_k / d_v / dtype combination outside the supported set */
     DELTALOG_ERR_CAP_RANGE = 3,         /* cap outside 1..64 */
-    DELTALOG_ERR_CUDA = 4               /* the CUDA runtime refused the launch or a copy */
+    DELTALOG_ERR_CUDA = 4,              /* the CUDA runtime refused the launch or a copy */
+    DELTALOG_ERR_STATIC_LIMIT = 5       /* the request does not fit the built-in staging area (see below) */
 };
 
 /* bits OR-ed into *status by kernels */
@@ -141,6 +142,35 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
                               const void *host_k, const void *host_v, const float *host_g,
                               const float *host_beta, const float *u_bonus,
                               const int32_t *slot_idx, int32_t B, void *host_out, void *stream);
+
+/*
+ * (No counterpart in the paper: a convenience for callers that must not allocate.)
+ *
+ * deltalog_decode_step_host without the staging argument.  Some callers cannot provide device
+ * staging buffers because they are not allowed to call cudaMalloc -- code that runs inside a
+ * latency-critical serving loop where an allocation may synchronise the device, plug-ins that are
+ * handed a stream but no allocator, or a process whose memory pool is owned by another component.
+ * For them the staging area is a fixed array inside the library (DELTALOG_STATIC_STAGING_BYTES of
+ * device memory on every GPU that loads the library, held until the process exits); this call
+ * allocates nothing, frees nothing and calls no allocating library routine.
+ *
+ *   - Limit: the staged tensors (q, k, v, g, beta, out, each rounded up to 256 bytes) must fit in
+ *     DELTALOG_STATIC_STAGING_BYTES; e.g. bf16, H = 32, d = 128 allows B <= 254 for GDN.  Larger
+ *     requests return DELTALOG_ERR_STATIC_LIMIT and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call before any stream capture begins.
+ *   - All calls on a device share the one array.  Two calls whose GPU work may overlap (different
+ *     streams, or a call issued before the previous host_out was consumed on another stream)
+ *     race on it; serialise them.  The array keeps the previous call's contents; the output part
+ *     is cleared at the start of every call, so rows the kernel skips (slot < 0, bad slot, full
+ *     log) read back as zeros in host_out.
+ *   - Arguments, results and return codes otherwise exactly as deltalog_decode_step_host.
+ */
+#define DELTALOG_STATIC_STAGING_BYTES (8u << 20)
+int deltalog_decode_step_host_static(const deltalog_desc *desc, const deltalog_state *state,
+                                     const void *host_q, const void *host_k, const void *host_v,
+                                     const float *host_g, const float *host_beta, const float *u_bonus,
+                                     const int32_t *slot_idx, int32_t B, void *host_out, void *stream);
 
 /* Human-readable text for a host return code (static storage). */
 const char *deltalog_status_string(int code);

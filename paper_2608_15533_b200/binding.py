@@ -17,7 +17,8 @@ import torch
 GDN, KDA, RWKV6 = 0, 1, 2
 F32, BF16 = 0, 1
 STATUS_LOG_FULL, STATUS_BAD_SLOT, STATUS_TIMEOUT = 1, 2, 4
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAP_RANGE, ERR_CUDA = 0, 1, 2, 3, 4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAP_RANGE, ERR_CUDA, ERR_STATIC_LIMIT = 0, 1, 2, 3, 4, 5
+STATIC_STAGING_BYTES = 8 << 20
 
 _TORCH_TO_DT = {torch.float32: F32, torch.bfloat16: BF16}
 _DT_TO_TORCH = {F32: torch.float32, BF16: torch.bfloat16}
@@ -26,6 +27,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
 
 EXPORTS = (
     "deltalog_decode_step", "deltalog_merge", "deltalog_eager_step", "deltalog_decode_step_host",
+    "deltalog_decode_step_host_static",
     "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
 )
 
@@ -72,6 +74,8 @@ def load_library() -> ctypes.CDLL:
         lib.deltalog_decode_step_host.restype = ctypes.c_int
         lib.deltalog_decode_step_host.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State),
                                                   ctypes.POINTER(_Staging)] + [vp] * 7 + [i32, vp, vp]
+        lib.deltalog_decode_step_host_static.restype = ctypes.c_int
+        lib.deltalog_decode_step_host_static.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State)] + [vp] * 7 + [i32, vp, vp]
         lib.deltalog_status_string.restype = ctypes.c_char_p
         lib.deltalog_status_string.argtypes = [ctypes.c_int]
         lib.deltalog_version.restype = ctypes.c_int
@@ -248,3 +252,19 @@ def decode_step_host(desc: Desc, state: State, staging: HostStaging, host_q, hos
         ctypes.byref(d), ctypes.byref(s), ctypes.byref(st), _ptr(host_q), _ptr(host_k), _ptr(host_v),
         _ptr(host_g), _ptr(host_beta), _ptr(u_bonus), _ptr(slot_idx), B, _ptr(host_out), _stream(stream))
     _check(rc, "deltalog_decode_step_host")
+
+
+def decode_step_host_static(desc: Desc, state: State, host_q, host_k, host_v, host_g, host_beta, host_out,
+                            u_bonus=None, slot_idx=None, stream=None) -> None:
+    """``deltalog_decode_step_host_static``: like ``decode_step_host`` but the device staging area is
+    the library's built-in array, for callers that must not allocate device memory.  Raises
+    ``DeltalogError`` (code ``ERR_STATIC_LIMIT``) when the token tensors exceed ``STATIC_STAGING_BYTES``.
+    Calls on one device share the array: do not let two of them overlap on the GPU."""
+    for t in (host_q, host_k, host_v, host_g, host_out):
+        assert t.device.type == "cpu"
+    B = host_q.shape[0]
+    d, s = desc.c_struct(), state.c_struct()
+    rc = load_library().deltalog_decode_step_host_static(
+        ctypes.byref(d), ctypes.byref(s), _ptr(host_q), _ptr(host_k), _ptr(host_v), _ptr(host_g),
+        _ptr(host_beta), _ptr(u_bonus), _ptr(slot_idx), B, _ptr(host_out), _stream(stream))
+    _check(rc, "deltalog_decode_step_host_static")

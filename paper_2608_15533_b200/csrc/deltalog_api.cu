@@ -283,6 +283,7 @@ const char *deltalog_status_string(int code) {
         case DELTALOG_ERR_UNSUPPORTED_SHAPE: return "unsupported shape or dtype combination";
         case DELTALOG_ERR_CAP_RANGE: return "log capacity outside 1..64";
         case DELTALOG_ERR_CUDA: return "CUDA runtime error";
+        case DELTALOG_ERR_STATIC_LIMIT: return "request larger than the built-in staging area (DELTALOG_STATIC_STAGING_BYTES)";
         default: return "unknown status code";
     }
 }

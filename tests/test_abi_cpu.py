@@ -29,8 +29,8 @@ def test_every_declared_symbol_is_exported(lib):
 def test_version_and_status_strings(lib):
     assert dl.version() >= 100
     assert dl.status_string(0) == "ok"
-    texts = {dl.status_string(c) for c in range(0, 6)}
-    assert len(texts) == 6 and "unknown status code" in texts
+    texts = {dl.status_string(c) for c in range(0, 7)}
+    assert len(texts) == 7 and "unknown status code" in texts
 
 
 def _desc(**kw):
