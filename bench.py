@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
 # captures summarised under profiles/ (bytes per (sequence, head) unit; None = not captured).
-NCU_DECODE_TRAFFIC_PER_UNIT = {}
+NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 73729.0, (2, 16): 78150.0, (3, 16): 21539.0}
 
 
 def measured_peak_gbs():
