@@ -198,31 +198,41 @@ def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int):
 
 def time_e2e_loop(rig: Rig, steps: int):
     """The same cycle through the host-buffer entry point: every step copies q, k, v, g, beta from
-    pinned host memory and reads the output back to pinned host memory."""
+    pinned host memory and reads the output back to pinned host memory.  Copy-in, kernel and
+    copy-out run on three streams over two staging sets (``deltalog_decode_step_host_overlapped``),
+    so the copies of step t+1 and t-1 overlap the kernel of step t."""
     dl, wl = rig.dl, rig.wl
-    staging = dl.HostStaging(rig.desc, wl.batch, rig.device)
+    streams = [torch.cuda.Stream(device=rig.device) for _ in range(3)]
+    sets = [(dl.HostStaging(rig.desc, wl.batch, rig.device), dl.HostLane(*streams),
+             torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()) for _ in range(2)]
     host_ring = [{k: (v.cpu().pin_memory() if v is not None else None) for k, v in tok.items()}
                  for tok in rig.rings[0]]
-    host_out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()
     rig.reset_logs()
+    torch.cuda.synchronize()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def run(n):
-        for t in range(n):
-            tok = host_ring[t % rig.RING]
-            dl.decode_step_host(rig.desc, rig.states[0], staging, tok["q"], tok["k"], tok["v"], tok["g"],
-                                tok["beta"], host_out, u_bonus=rig.bonus[0], slot_idx=rig.slot_idx)
-            if (t + 1) % rig.cap == 0:
-                rig.merge(0)
+        with torch.cuda.stream(streams[1]):  # merges go to the compute stream
+            for t in range(n):
+                tok = host_ring[t % rig.RING]
+                staging, lane, host_out = sets[t % 2]
+                dl.decode_step_host_overlapped(rig.desc, rig.states[0], staging, lane, tok["q"], tok["k"], tok["v"],
+                                               tok["g"], tok["beta"], host_out, u_bonus=rig.bonus[0],
+                                               slot_idx=rig.slot_idx)
+                if (t + 1) % rig.cap == 0:
+                    rig.merge(0)
 
     run(rig.cap)  # warm the copy path, ends on a merge
     launch.barrier()
     torch.cuda.synchronize()
-    start.record()
+    start.record(streams[1])
     run(steps)
-    end.record()
+    for st in streams:
+        st.synchronize()
+    end.record(streams[1])
     torch.cuda.synchronize()
     launch.barrier()
+    staging = sets[0][0]
     return start.elapsed_time(end), staging.h2d_bytes(rig.desc), staging.d2h_bytes()
 
 

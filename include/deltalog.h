@@ -144,6 +144,33 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
                               const int32_t *slot_idx, int32_t B, void *host_out, void *stream);
 
 /*
+ * deltalog_decode_step_host with the three phases of a step on three streams, so that the copies
+ * of consecutive steps overlap the kernels: while step t runs on compute_stream, the token tensors
+ * of step t+1 are already being copied in and the output of step t-1 is being copied out.  The
+ * caller owns the streams and the events and alternates between (at least) two sets of
+ * {staging, in_done, compute_done, out_done}; the streams are shared by all sets.  Per call:
+ *     copy_in_stream :  wait compute_done (the kernel that last read this staging set);  H2D copies
+ *                       of q, k, v, g, beta;  record in_done
+ *     compute_stream :  wait in_done and out_done (previous read-back of this set);  decode kernel;
+ *                       record compute_done
+ *     copy_out_stream:  wait compute_done;  D2H copy of out into host_out;  record out_done
+ * Kernels of consecutive steps (and the caller's deltalog_merge calls, which belong on
+ * compute_stream) stay ordered because they share compute_stream.  Synchronise out_done before
+ * reading host_out.  Events must have been created by the caller; an event that was never recorded
+ * is treated as complete.  Other arguments and return codes as deltalog_decode_step_host.
+ */
+typedef struct {
+    void *copy_in_stream, *compute_stream, *copy_out_stream; /* cudaStream_t */
+    void *in_done, *compute_done, *out_done;                 /* cudaEvent_t, one triple per staging set */
+} deltalog_host_lane;
+
+int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltalog_state *state,
+                                         const deltalog_staging *staging, const deltalog_host_lane *lane,
+                                         const void *host_q, const void *host_k, const void *host_v,
+                                         const float *host_g, const float *host_beta, const float *u_bonus,
+                                         const int32_t *slot_idx, int32_t B, void *host_out);
+
+/*
  * (No counterpart in the paper: a convenience for callers that must not allocate.)
  *
  * deltalog_decode_step_host without the staging argument.  Some callers cannot provide device

@@ -27,7 +27,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
 
 EXPORTS = (
     "deltalog_decode_step", "deltalog_merge", "deltalog_eager_step", "deltalog_decode_step_host",
-    "deltalog_decode_step_host_static",
+    "deltalog_decode_step_host_static", "deltalog_decode_step_host_overlapped",
     "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
 )
 
@@ -50,6 +50,11 @@ class _State(ctypes.Structure):
 
 class _Staging(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("q", "k", "v", "g", "beta", "out")]
+
+
+class _Lane(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("copy_in_stream", "compute_stream", "copy_out_stream", "in_done", "compute_done", "out_done")]
 
 
 _lib = None
@@ -76,6 +81,9 @@ def load_library() -> ctypes.CDLL:
                                                   ctypes.POINTER(_Staging)] + [vp] * 7 + [i32, vp, vp]
         lib.deltalog_decode_step_host_static.restype = ctypes.c_int
         lib.deltalog_decode_step_host_static.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State)] + [vp] * 7 + [i32, vp, vp]
+        lib.deltalog_decode_step_host_overlapped.restype = ctypes.c_int
+        lib.deltalog_decode_step_host_overlapped.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State),
+                                                             ctypes.POINTER(_Staging), ctypes.POINTER(_Lane)] + [vp] * 7 + [i32, vp]
         lib.deltalog_status_string.restype = ctypes.c_char_p
         lib.deltalog_status_string.argtypes = [ctypes.c_int]
         lib.deltalog_version.restype = ctypes.c_int
@@ -268,3 +276,28 @@ def decode_step_host_static(desc: Desc, state: State, host_q, host_k, host_v, ho
         ctypes.byref(d), ctypes.byref(s), _ptr(host_q), _ptr(host_k), _ptr(host_v), _ptr(host_g),
         _ptr(host_beta), _ptr(u_bonus), _ptr(slot_idx), B, _ptr(host_out), _stream(stream))
     _check(rc, "deltalog_decode_step_host_static")
+
+
+class HostLane:
+    """Streams (shared) and one event triple (per staging set) for ``decode_step_host_overlapped``."""
+
+    def __init__(self, copy_in: "torch.cuda.Stream", compute: "torch.cuda.Stream", copy_out: "torch.cuda.Stream"):
+        self.copy_in, self.compute, self.copy_out = copy_in, compute, copy_out
+        self.in_done, self.compute_done, self.out_done = (torch.cuda.Event() for _ in range(3))
+        for ev, st in ((self.in_done, copy_in), (self.compute_done, compute), (self.out_done, copy_out)):
+            ev.record(st)  # creates the underlying CUDA event
+
+    def c_struct(self) -> _Lane:
+        return _Lane(self.copy_in.cuda_stream, self.compute.cuda_stream, self.copy_out.cuda_stream,
+                     self.in_done.cuda_event, self.compute_done.cuda_event, self.out_done.cuda_event)
+
+
+def decode_step_host_overlapped(desc: Desc, state: State, staging: HostStaging, lane: HostLane, host_q, host_k,
+                                host_v, host_g, host_beta, host_out, u_bonus=None, slot_idx=None) -> None:
+    """``deltalog_decode_step_host_overlapped``: copy-in, kernel and copy-out on the lane's three streams."""
+    B = host_q.shape[0]
+    d, s, st, ln = desc.c_struct(), state.c_struct(), staging.c_struct(), lane.c_struct()
+    rc = load_library().deltalog_decode_step_host_overlapped(
+        ctypes.byref(d), ctypes.byref(s), ctypes.byref(st), ctypes.byref(ln), _ptr(host_q), _ptr(host_k),
+        _ptr(host_v), _ptr(host_g), _ptr(host_beta), _ptr(u_bonus), _ptr(slot_idx), B, _ptr(host_out))
+    _check(rc, "deltalog_decode_step_host_overlapped")

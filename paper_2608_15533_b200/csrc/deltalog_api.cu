@@ -276,6 +276,54 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
     return DELTALOG_OK;
 }
 
+int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltalog_state *state,
+                                         const deltalog_staging *staging, const deltalog_host_lane *lane,
+                                         const void *host_q, const void *host_k, const void *host_v,
+                                         const float *host_g, const float *host_beta, const float *u_bonus,
+                                         const int32_t *slot_idx, int32_t B, void *host_out) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (!staging || !lane || !host_q || !host_k || !host_v || !host_g || !host_out) return DELTALOG_ERR_INVALID_ARG;
+    if (!lane->in_done || !lane->compute_done || !lane->out_done) return DELTALOG_ERR_INVALID_ARG;
+    if (desc->op != DELTALOG_RWKV6 && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
+    if (!staging->q || !staging->k || !staging->v || !staging->g || !staging->out) return DELTALOG_ERR_INVALID_ARG;
+    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
+    if (B == 0) return DELTALOG_OK;
+    cudaStream_t s_in = static_cast<cudaStream_t>(lane->copy_in_stream);
+    cudaStream_t s_cmp = static_cast<cudaStream_t>(lane->compute_stream);
+    cudaStream_t s_out = static_cast<cudaStream_t>(lane->copy_out_stream);
+    cudaEvent_t e_in = static_cast<cudaEvent_t>(lane->in_done);
+    cudaEvent_t e_cmp = static_cast<cudaEvent_t>(lane->compute_done);
+    cudaEvent_t e_out = static_cast<cudaEvent_t>(lane->out_done);
+    const size_t units = (size_t)B * desc->H;
+    const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
+    const size_t vec = units * desc->d_k * esz;
+    const size_t gbytes = units * (desc->op == DELTALOG_GDN ? 1 : desc->d_k) * sizeof(float);
+    // copy-in stream: the staging inputs are free once the kernel that last read them is done
+    bool ok = cudaStreamWaitEvent(s_in, e_cmp, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    if (desc->op != DELTALOG_RWKV6)
+        ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s_in) ==
+                       cudaSuccess;
+    ok = ok && cudaEventRecord(e_in, s_in) == cudaSuccess;
+    // compute stream: inputs landed, and the previous output of this staging set has been read back
+    ok = ok && cudaStreamWaitEvent(s_cmp, e_in, 0) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(s_cmp, e_out, 0) == cudaSuccess;
+    if (!ok) return DELTALOG_ERR_CUDA;
+    if (int rc = deltalog_decode_step(desc, state, staging->q, staging->k, staging->v, staging->g,
+                                      staging->beta, u_bonus, slot_idx, B, staging->out, lane->compute_stream))
+        return rc;
+    ok = cudaEventRecord(e_cmp, s_cmp) == cudaSuccess;
+    // copy-out stream
+    ok = ok && cudaStreamWaitEvent(s_out, e_cmp, 0) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(host_out, staging->out, units * desc->d_v * esz, cudaMemcpyDeviceToHost, s_out) ==
+                   cudaSuccess;
+    ok = ok && cudaEventRecord(e_out, s_out) == cudaSuccess;
+    return ok ? DELTALOG_OK : DELTALOG_ERR_CUDA;
+}
+
 const char *deltalog_status_string(int code) {
     switch (code) {
         case DELTALOG_OK: return "ok";

@@ -335,3 +335,38 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         torch.cuda.synchronize()
         assert torch.equal(out.cpu(), host_out)
     assert torch.equal(s_dev.U_log, s_host.U_log)
+
+
+def test_overlapped_host_entry_point_matches_device_entry_point_over_a_cycle():
+    """Three streams, two staging sets, merges on the compute stream: same bits as the plain path."""
+    import paper_2608_15533_b200 as dl
+
+    wl = small(KDA, 128, torch.bfloat16, batch=4, H=2)
+    src = workloads.TokenSource(wl)
+    S0 = src.initial_state().to(DEV)
+    desc = make_desc(wl, 4)
+    s_dev, s_host = dl.State(desc, S0.clone()), dl.State(desc, S0.clone())
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    sets = [(dl.HostStaging(desc, wl.batch, DEV), dl.HostLane(*streams)) for _ in range(2)]
+    toks = [src.token() for _ in range(10)]
+    pinned = [{k_: v_.pin_memory() for k_, v_ in tok.items()} for tok in toks]
+    host_outs = [torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory() for _ in toks]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(streams[1]):
+        for t, p in enumerate(pinned):
+            staging, lane = sets[t % 2]
+            dl.decode_step_host_overlapped(desc, s_host, staging, lane, p["q"], p["k"], p["v"], p["g"], p["beta"],
+                                           host_outs[t])
+            if (t + 1) % 4 == 0:
+                dl.merge(desc, s_host, only_if_full=True)
+    for st in streams:
+        st.synchronize()
+    for t, tok in enumerate(toks):
+        dev = {k_: v_.to(DEV) for k_, v_ in tok.items()}
+        out = dl.decode_step(desc, s_dev, dev["q"], dev["k"], dev["v"], dev["g"], beta=dev["beta"])
+        if (t + 1) % 4 == 0:
+            dl.merge(desc, s_dev, only_if_full=True)
+        assert torch.equal(out.cpu(), host_outs[t]), f"step {t}"
+    torch.cuda.synchronize()
+    assert torch.equal(s_dev.S_base, s_host.S_base) and torch.equal(s_dev.U_log, s_host.U_log)
+    assert torch.equal(s_dev.log_len, s_host.log_len)
