@@ -69,11 +69,12 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
 
-// Cooperative async copy of `bytes` (multiple of 16) by the whole CTA.
-__device__ __forceinline__ void cta_cp_async(void *smem_dst, const void *gmem_src, int bytes, int tid) {
+// Cooperative async copy of `bytes` (multiple of 16) by the whole CTA of `nthreads` threads.
+__device__ __forceinline__ void cta_cp_async(void *smem_dst, const void *gmem_src, int bytes, int tid,
+                                             int nthreads = kThreads) {
     char *d = static_cast<char *>(smem_dst);
     const char *s = static_cast<const char *>(gmem_src);
-    for (int off = tid * 16; off < bytes; off += kThreads * 16) cp_async16(d + off, s + off);
+    for (int off = tid * 16; off < bytes; off += nthreads * 16) cp_async16(d + off, s + off);
 }
 
 __device__ __forceinline__ float4 fma4(float a, const float4 &x, const float4 &acc) {

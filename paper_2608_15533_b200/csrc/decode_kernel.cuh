@@ -17,14 +17,22 @@
 
 namespace deltalog {
 
+// Threads per CTA: 256 at head size 128; 128 at head size 64, where the tile is only 16 KiB and the
+// run time of a CTA is one long latency chain (length -> snapshot and log -> coefficients): smaller
+// CTAs let eight of them overlap their chains on an SM instead of four.
+template <int D>
+__host__ __device__ constexpr int decode_threads() {
+    return D >= 128 ? 256 : 128;
+}
+
 template <int D, typename IO, typename UL>
-constexpr size_t decode_smem_bytes(int op, int cap) {
+__host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
     const size_t dl = (op == DELTALOG_GDN) ? 1 : D;
     size_t bytes = 0;
     bytes += sizeof(float) * D * 5;                 // q, k (raw), mul_k, mul_q, lbar'/u scratch
     bytes += sizeof(float) * D;                     // lbar_old (vector ops)
     bytes += sizeof(float) * 2 * kMaxCap;           // replay coefficients
-    bytes += sizeof(float) * 2 * D * (kThreads / (D / 4));  // cross-row-lane partial sums
+    bytes += sizeof(float) * 2 * D * (decode_threads<D>() / (D / 4));  // cross-row-lane partial sums
     bytes += 16;                                    // scalars
     bytes += sizeof(UL) * (size_t)cap * D;          // U log
     bytes += sizeof(IO) * (size_t)cap * D;          // K log
@@ -33,12 +41,14 @@ constexpr size_t decode_smem_bytes(int op, int cap) {
 }
 
 template <int OP, int D, typename IO, typename UL>
-__global__ void __launch_bounds__(kThreads, 2) decode_append_kernel(StateArgs st, TokenArgs tk) {
+__global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? 2 : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
+    constexpr int NT = decode_threads<D>();
+    constexpr int NW = NT / 32;
     constexpr bool kDelta = (OP != DELTALOG_RWKV6);
     constexpr bool kVecDecay = (OP != DELTALOG_GDN);
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4;          // float4 columns per state row
-    constexpr int RL = kThreads / C4;  // rows covered by one pass of the CTA
+    constexpr int RL = NT / C4;        // rows covered by one pass of the CTA
     constexpr int NP = D / RL;         // passes over the tile
     constexpr int EPL = D / 32;        // key elements per lane in a warp-wide dot product
 
@@ -82,9 +92,9 @@ __global__ void __launch_bounds__(kThreads, 2) decode_append_kernel(StateArgs st
     const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
     const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
     const float *Lg = st.decay_log + unit * cap * DL;
-    cta_cp_async(K_s, Kg, len * D * (int)sizeof(IO), tid);
-    cta_cp_async(U_s, Ug, len * D * (int)sizeof(UL), tid);
-    if (kVecDecay) cta_cp_async(Lam_s, Lg, len * D * (int)sizeof(float), tid);
+    cta_cp_async(K_s, Kg, len * D * (int)sizeof(IO), tid, NT);
+    cta_cp_async(U_s, Ug, len * D * (int)sizeof(UL), tid, NT);
+    if (kVecDecay) cta_cp_async(Lam_s, Lg, len * D * (int)sizeof(float), tid, NT);
     cp_async_commit();
     if (!kVecDecay && tid < len) Lam_s[tid] = Lg[tid];
 
@@ -111,7 +121,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_append_kernel(StateArgs st
     __syncthreads();
 
     // ---- 3. key-side replay coefficients: one warp per live entry ---------------------------
-    for (int i = warp; i < len; i += kWarps) {
+    for (int i = warp; i < len; i += NW) {
         float dq = 0.f, dk = 0.f;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
@@ -129,7 +139,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_append_kernel(StateArgs st
             if (kDelta) ck_s[i] = w * dk;
         }
     }
-    if (warp == kWarps - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
+    if (warp == NW - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
         float d = 0.f;
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {

@@ -151,7 +151,7 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
     auto kernel = decode_append_kernel<OP, D, IO, UL>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<total, kThreads, smem, stream>>>(st, tk);
+    kernel<<<total, decode_threads<D>(), smem, stream>>>(st, tk);
     return finish_launch();
 }
 
