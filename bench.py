@@ -151,47 +151,108 @@ class Rig:
 
 
 def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
-    """Time exactly ``steps`` steps (decode every step, merge after every cap-th) on the current
-    stream; returns total ms, summed decode-kernel ms and summed merge-kernel ms."""
+    """Time exactly ``steps`` steps (decode every step, merge after every cap-th) as plain launches
+    on the current stream.  With ``per_kernel`` two events per cycle split the time into decode
+    launches and the merge launch (an event between every pair of launches would itself cost
+    several microseconds per step); returns total ms, summed decode ms, summed merge ms, merges."""
     cap = rig.cap
     ev = lambda: torch.cuda.Event(enable_timing=True)
     start, end = ev(), ev()
-    d0 = [ev() for _ in range(steps)] if per_kernel else None
-    d1 = [ev() for _ in range(steps)] if per_kernel else None
-    m1 = {}
+    marks = []  # (event before the first decode of a cycle, event after its last decode, event after its merge)
     launch.barrier()
     torch.cuda.synchronize()
     start.record()
     for t in range(steps):
         for layer in range(rig.layers):
-            if per_kernel and layer == 0:
-                d0[t].record()
+            if per_kernel and layer == 0 and t % cap == 0:
+                marks.append([ev(), None, None])
+                marks[-1][0].record()
             rig.decode(t, layer)
-            if per_kernel and layer == 0:
-                d1[t].record()
             if (t + 1) % cap == 0:
+                if per_kernel and layer == 0:
+                    marks[-1][1] = ev(); marks[-1][1].record()
                 rig.merge(layer)
                 if per_kernel and layer == 0:
-                    m1[t] = ev(); m1[t].record()
+                    marks[-1][2] = ev(); marks[-1][2].record()
     end.record()
     torch.cuda.synchronize()
     launch.barrier()
     total = start.elapsed_time(end)
-    dec = sum(a.elapsed_time(b) for a, b in zip(d0, d1)) if per_kernel else None
-    mrg = sum(d1[t].elapsed_time(e) for t, e in m1.items()) if per_kernel else None
-    return total, dec, mrg, len(m1)
+    full = [m for m in marks if m[2] is not None]
+    dec = sum(a.elapsed_time(b) for a, b, _ in full) if per_kernel else None
+    mrg = sum(b.elapsed_time(c) for _, b, c in full) if per_kernel else None
+    return total, dec, mrg, len(full)
 
 
-def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int):
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    dl = rig.dl
+def graph_steps(cap: int) -> int:
+    """Steps per captured graph: whole cycles that also return to the start of the token ring."""
+    import math
+
+    return cap * Rig.RING // math.gcd(cap, Rig.RING)
+
+
+def time_graph_loop(rig: Rig, steps: int):
+    """Time exactly ``steps`` steps replayed from one CUDA graph that holds ``graph_steps`` steps
+    (decode launches and the merge launches between them), the way a serving loop would run the
+    cycle.  ``steps`` must be a multiple of the graph length.  Returns total ms."""
+    g_len = graph_steps(rig.cap)
+    assert steps % g_len == 0
+    stream = torch.cuda.Stream(device=rig.device)
+    graph = torch.cuda.CUDAGraph()
     torch.cuda.synchronize()
-    start.record()
-    for t in range(steps):
-        tok = rig.rings[0][t % rig.RING]
-        dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
-                      u_bonus=rig.bonus[0], out=rig.out)
-    end.record()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for t in range(g_len):
+                for layer in range(rig.layers):
+                    rig.decode(t, layer)
+                    if (t + 1) % rig.cap == 0:
+                        rig.merge(layer)
+        graph.replay()  # warm the replay path once (a whole number of cycles: the logs end empty)
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launch.barrier()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        start.record()
+        for _ in range(steps // g_len):
+            graph.replay()
+        end.record()
+    torch.cuda.synchronize()
+    launch.barrier()
+    return start.elapsed_time(end)
+
+
+def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = True):
+    """The eager dense comparator on the same token ring, launched the same way as the main loop."""
+    dl = rig.dl
+
+    def launch_steps(n):
+        for t in range(n):
+            tok = rig.rings[0][t % rig.RING]
+            dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                          u_bonus=rig.bonus[0], out=rig.out)
+
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    use_graph = use_graph and steps % rig.RING == 0
+    stream = torch.cuda.Stream(device=rig.device) if use_graph else torch.cuda.current_stream()
+    graph = None
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        if use_graph:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                launch_steps(rig.RING)
+            graph.replay()
+        else:
+            launch_steps(rig.RING)
+        torch.cuda.synchronize()
+        start.record()
+        if use_graph:
+            for _ in range(steps // rig.RING):
+                graph.replay()
+        else:
+            launch_steps(steps)
+        end.record()
     torch.cuda.synchronize()
     return start.elapsed_time(end)
 
@@ -297,6 +358,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
     ap.add_argument("--cap", type=int, default=16, help="log capacity of the headline number")
+    ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--no-extras", action="store_true", help="skip the capacity sweep, eager and CPU legs")
     ap.add_argument("--only-hot-loop", action="store_true",
                     help="warm-up and timed loop only (for profiler captures)")
@@ -333,10 +395,18 @@ def main():
     if args.only_hot_loop:
         time_cycle_loop(rig, args.steps, per_kernel=False)
         return launch.finalize()
+    use_graph = (not args.no_graph) and args.steps % graph_steps(cap) == 0
     with ClockSampler(local) as clocks:
         l0 = dl.launch_count()
-        total_ms, dec_ms, mrg_ms, n_merges = time_cycle_loop(rig, args.steps)
-        gpu_launches = dl.launch_count() - l0
+        if use_graph:
+            total_ms = time_graph_loop(rig, args.steps)
+            # kernels executed by the replays (the host-side counter only sees the capture)
+            gpu_launches = layers * (args.steps + args.steps // cap)
+        else:
+            total_ms, _, _, _ = time_cycle_loop(rig, args.steps, per_kernel=False)
+            gpu_launches = dl.launch_count() - l0
+        # same steps again as plain launches with two events per cycle: the split into decode and merge time
+        split_ms, dec_ms, mrg_ms, n_merges = time_cycle_loop(rig, args.steps)
     assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
     total_ms = launch.max_over_ranks(total_ms, device)
     all_units = launch.sum_over_ranks(units * layers, device)
@@ -347,7 +417,7 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     fills = [t % cap for t in range(args.steps)]
     dec_bytes = statistics.mean(traffic.decode_read(u, f) + traffic.decode_write(u) for f in fills) * units
-    dec_ms_avg = dec_ms / args.steps
+    dec_ms_avg = dec_ms / (n_merges * cap) if n_merges else float("nan")
     achieved = dec_bytes / (dec_ms_avg * 1e-3) / 1e9
     traffic_ncu = NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
     line = {
@@ -358,6 +428,7 @@ def main():
             "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
             "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
             "io": str(wl.io_dtype).replace("torch.", ""), "merge": f"after every {cap}th step",
+            "launch": (f"one CUDA graph of {graph_steps(cap)} steps, replayed" if use_graph else "plain launches"),
             "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
             "parallelism": f"rows sharded over {size} GPU(s), no collective",
         },
@@ -374,6 +445,7 @@ def main():
             "hbm_gbs": cyc["total"] * all_units / (ms_per_step * 1e-3) / 1e9,
             "bytes_written_per_unit_step": cyc["write"], "write_reduction_vs_eager": cyc["write_reduction"],
             "decode_ms_per_step": dec_ms_avg, "merge_ms_per_merge": (mrg_ms / n_merges) if n_merges else None,
+            "plain_launch_ms_per_step": split_ms / args.steps,
         },
     }
     line["amortized"]["frac_of_nominal_8TBs"] = line["amortized"]["hbm_gbs"] / NOMINAL_HBM_GBS / size
@@ -391,8 +463,7 @@ def main():
         # eager dense comparator on the same inputs
         rig.reset_logs()
         S = rig.states[0].S_base
-        time_eager_loop(rig, S, 8)
-        eager_ms = time_eager_loop(rig, S, args.steps) / args.steps
+        eager_ms = time_eager_loop(rig, S, args.steps, use_graph) / args.steps
         eager_bytes = (traffic.eager_read(u) + traffic.eager_write(u)) * units
         line["eager_kernel"] = {"ms_per_step": eager_ms, "value": units / (eager_ms * 1e-3),
                                 "hbm_gbs": eager_bytes / (eager_ms * 1e-3) / 1e9,
@@ -415,7 +486,8 @@ def main():
                 if (t + 1) % c == 0:
                     rig.merge()
             rig.reset_logs()
-            ms, _, _, _ = time_cycle_loop(rig, args.steps, per_kernel=False)
+            ms = time_graph_loop(rig, args.steps) if use_graph and args.steps % graph_steps(c) == 0 else \
+                time_cycle_loop(rig, args.steps, per_kernel=False)[0]
             cc = traffic.cycle_bytes(u, c)
             sweep[str(c)] = {"ms_per_step": ms / args.steps, "value": units * args.steps / (ms * 1e-3),
                              "write_reduction_vs_eager": cc["write_reduction"],

@@ -40,8 +40,11 @@ __host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
     return bytes;
 }
 
+#ifndef DELTALOG_SIMPLE_CTAS
+#define DELTALOG_SIMPLE_CTAS 2
+#endif
 template <int OP, int D, typename IO, typename UL>
-__global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? 2 : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
+__global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPLE_CTAS : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
     constexpr int NT = decode_threads<D>();
     constexpr int NW = NT / 32;
     constexpr bool kDelta = (OP != DELTALOG_RWKV6);
