@@ -130,7 +130,10 @@ class Rig:
             self.rings.append([src.token() for _ in range(self.RING)])
         self.out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
         self.slot_idx = None
-        self.step_slots = None   # optional per-step slot lists (staggered start)
+        self.staggered = bool(wl.staggered)
+        if self.staggered:  # serving shape: rows address a shuffled slot pool, every row at its own log fill
+            self.slot_idx = workloads.slot_permutation(wl).to(device)
+            self.delay = ((cap - workloads.fill_offsets(wl, cap)) % cap).to(device)
 
     def decode(self, t, layer=0, slot_idx=None):
         tok = self.rings[layer][t % self.RING]
@@ -138,13 +141,35 @@ class Rig:
                             beta=tok["beta"], u_bonus=self.bonus[layer],
                             slot_idx=self.slot_idx if slot_idx is None else slot_idx, out=self.out)
 
-    def merge(self, layer=0, only_if_full=True):
+    def merge(self, layer=0, only_if_full=None):
+        if only_if_full is None:   # a uniform batch folds every row at once; a staggered one uses the predicate
+            only_if_full = self.staggered
         self.dl.merge(self.desc, self.states[layer], slot_idx=self.slot_idx, n=self.wl.batch,
                       only_if_full=only_if_full)
 
+    def step(self, t, layer=0):
+        """One step of the hot path for one layer.  Uniform batch: decode, and the merge after every
+        cap-th step.  Staggered batch: a predicate merge over the whole batch (only full logs fold,
+        about 1/cap of the rows per step), then decode."""
+        if self.staggered:
+            self.merge(layer, only_if_full=True)
+            self.decode(t, layer)
+        else:
+            self.decode(t, layer)
+            if (t + 1) % self.cap == 0:
+                self.merge(layer)
+
     def reset_logs(self):
+        """Fold everything; a staggered batch is then rolled forward so that row b holds
+        (cap - delay_b) entries: rows sit out (slot -1) until their start step, real decode steps
+        fill the logs (nothing is fabricated)."""
         for layer in range(self.layers):
             self.merge(layer, only_if_full=False)
+        if self.staggered:
+            for t in range(self.cap):
+                slots = torch.where(self.delay <= t, self.slot_idx, torch.full_like(self.slot_idx, -1))
+                for layer in range(self.layers):
+                    self.decode(t, layer, slot_idx=slots)
 
     def status(self):
         return [int(s.status.item()) for s in self.states]
@@ -164,6 +189,17 @@ def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
     start.record()
     for t in range(steps):
         for layer in range(rig.layers):
+            if rig.staggered:
+                if per_kernel and layer == 0:  # one layer in `layers` carries the events
+                    marks.append([ev(), ev(), ev()])
+                    marks[-1][1].record()       # merge first here: [1] -> merge -> [2]=[0] -> decode -> end
+                    rig.merge(layer, only_if_full=True)
+                    marks[-1][0].record()
+                    rig.decode(t, layer)
+                    marks[-1][2].record()
+                else:
+                    rig.step(t, layer)
+                continue
             if per_kernel and layer == 0 and t % cap == 0:
                 marks.append([ev(), None, None])
                 marks[-1][0].record()
@@ -179,23 +215,28 @@ def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
     launch.barrier()
     total = start.elapsed_time(end)
     full = [m for m in marks if m[2] is not None]
-    dec = sum(a.elapsed_time(b) for a, b, _ in full) if per_kernel else None
-    mrg = sum(b.elapsed_time(c) for _, b, c in full) if per_kernel else None
+    if rig.staggered:  # per step: [1] merge [0] decode [2]
+        dec = sum(a.elapsed_time(c) for a, _, c in full) if per_kernel else None
+        mrg = sum(b.elapsed_time(a) for a, b, _ in full) if per_kernel else None
+    else:              # per cycle: [0] cap decodes [1] merge [2]
+        dec = sum(a.elapsed_time(b) for a, b, _ in full) if per_kernel else None
+        mrg = sum(b.elapsed_time(c) for _, b, c in full) if per_kernel else None
     return total, dec, mrg, len(full)
 
 
-def graph_steps(cap: int) -> int:
-    """Steps per captured graph: whole cycles that also return to the start of the token ring."""
+def graph_steps(cap: int, staggered: bool = False) -> int:
+    """Steps per captured graph: whole cycles that also return to the start of the token ring (a
+    staggered batch launches the same two kernels every step, so the ring length is enough)."""
     import math
 
-    return cap * Rig.RING // math.gcd(cap, Rig.RING)
+    return Rig.RING if staggered else cap * Rig.RING // math.gcd(cap, Rig.RING)
 
 
 def time_graph_loop(rig: Rig, steps: int):
     """Time exactly ``steps`` steps replayed from one CUDA graph that holds ``graph_steps`` steps
     (decode launches and the merge launches between them), the way a serving loop would run the
     cycle.  ``steps`` must be a multiple of the graph length.  Returns total ms."""
-    g_len = graph_steps(rig.cap)
+    g_len = graph_steps(rig.cap, rig.staggered)
     assert steps % g_len == 0
     stream = torch.cuda.Stream(device=rig.device)
     graph = torch.cuda.CUDAGraph()
@@ -204,10 +245,9 @@ def time_graph_loop(rig: Rig, steps: int):
         with torch.cuda.graph(graph, stream=stream):
             for t in range(g_len):
                 for layer in range(rig.layers):
-                    rig.decode(t, layer)
-                    if (t + 1) % rig.cap == 0:
-                        rig.merge(layer)
-        graph.replay()  # warm the replay path once (a whole number of cycles: the logs end empty)
+                    rig.step(t, layer)
+        for _ in range(2 if rig.staggered else 1):  # warm the replay path; an unstaggered graph ends on empty logs,
+            graph.replay()                         # a staggered batch of ring-length graphs needs cap steps per period
     torch.cuda.synchronize()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launch.barrier()
@@ -274,14 +314,16 @@ def time_e2e_loop(rig: Rig, steps: int):
 
     def run(n):
         with torch.cuda.stream(streams[1]):  # merges go to the compute stream
+            if rig.staggered:
+                rig.merge(0)   # rows whose log is full fold before the first decode
             for t in range(n):
                 tok = host_ring[t % rig.RING]
                 staging, lane, host_out = sets[t % 2]
                 dl.decode_step_host_overlapped(rig.desc, rig.states[0], staging, lane, tok["q"], tok["k"], tok["v"],
                                                tok["g"], tok["beta"], host_out, u_bonus=rig.bonus[0],
                                                slot_idx=rig.slot_idx)
-                if (t + 1) % rig.cap == 0:
-                    rig.merge(0)
+                if rig.staggered or (t + 1) % rig.cap == 0:
+                    rig.merge(0)   # predicate merge: after the step here, i.e. before the next decode
 
     run(rig.cap)  # warm the copy path, ends on a merge
     launch.barrier()
@@ -356,7 +398,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2048)
     ap.add_argument("--warmup", type=int, default=256)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3])
+    ap.add_argument("--config", type=int, default=1, choices=[1, 2, 3, 4])
     ap.add_argument("--cap", type=int, default=16, help="log capacity of the headline number")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--no-extras", action="store_true", help="skip the capacity sweep, eager and CPU legs")
@@ -377,31 +419,31 @@ def main():
     warmup = max(args.warmup, 3)
     layers = wl.layers
     rig = Rig(wl, cap, device, seed_offset=rank, layers=layers)
-    if wl.staggered:
-        rig.slot_idx = workloads.slot_permutation(wl).to(device)
+    stag = rig.staggered
+    g_len = graph_steps(cap, stag)
     u = unit_shape(wl)
     units = wl.units
 
     # ---- warm-up, then the timed region: exactly K steps ---------------------------------------
     launches0 = dl.launch_count()
+    rig.reset_logs()
     for t in range(warmup):
         for layer in range(layers):
-            rig.decode(t, layer)
-            if (t + 1) % cap == 0:
-                rig.merge(layer)
-    rig.reset_logs()
+            rig.step(t, layer)
+    if not stag:
+        rig.reset_logs()   # a uniform batch starts the timed region on empty logs
     torch.cuda.synchronize()
     warm_launches = dl.launch_count() - launches0
     if args.only_hot_loop:
         time_cycle_loop(rig, args.steps, per_kernel=False)
         return launch.finalize()
-    use_graph = (not args.no_graph) and args.steps % graph_steps(cap) == 0
+    use_graph = (not args.no_graph) and args.steps % g_len == 0
     with ClockSampler(local) as clocks:
         l0 = dl.launch_count()
         if use_graph:
             total_ms = time_graph_loop(rig, args.steps)
             # kernels executed by the replays (the host-side counter only sees the capture)
-            gpu_launches = layers * (args.steps + args.steps // cap)
+            gpu_launches = layers * (2 * args.steps if stag else args.steps + args.steps // cap)
         else:
             total_ms, _, _, _ = time_cycle_loop(rig, args.steps, per_kernel=False)
             gpu_launches = dl.launch_count() - l0
@@ -417,7 +459,8 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     fills = [t % cap for t in range(args.steps)]
     dec_bytes = statistics.mean(traffic.decode_read(u, f) + traffic.decode_write(u) for f in fills) * units
-    dec_ms_avg = dec_ms / (n_merges * cap) if n_merges else float("nan")
+    # events bracket cap decode launches per mark in a uniform batch, one decode launch per mark in a staggered one
+    dec_ms_avg = dec_ms / (n_merges * (1 if stag else cap)) if n_merges else float("nan")
     achieved = dec_bytes / (dec_ms_avg * 1e-3) / 1e9
     traffic_ncu = NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
     line = {
@@ -427,8 +470,9 @@ def main():
         "config": {
             "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
             "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
-            "io": str(wl.io_dtype).replace("torch.", ""), "merge": f"after every {cap}th step",
-            "launch": (f"one CUDA graph of {graph_steps(cap)} steps, replayed" if use_graph else "plain launches"),
+            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("predicate merge over the batch before every step, fills staggered over 0..cap-1" if stag
+                      else f"after every {cap}th step"),
+            "launch": (f"one CUDA graph of {g_len} steps, replayed" if use_graph else "plain launches"),
             "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
             "parallelism": f"rows sharded over {size} GPU(s), no collective",
         },

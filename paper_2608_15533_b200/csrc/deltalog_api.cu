@@ -159,10 +159,19 @@ template <int OP, int D, typename IO>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
     using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
-    auto kernel = merge_kernel<OP, D, IO, UL>;
     const size_t smem = merge_smem_bytes<D>(st.cap);
-    if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<n * st.H, kThreads, smem, stream>>>(st, slot_idx, only_if_full);
+    // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
+    // call over a whole batch whose fills are staggered) most units are skipped: eight per CTA.
+    const int pairs = n * st.H;
+    if (only_if_full) {
+        auto kernel = merge_kernel<OP, D, IO, UL, 8>;
+        if (int rc = ensure_smem(kernel, smem)) return rc;
+        kernel<<<(pairs + 7) / 8, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
+    } else {
+        auto kernel = merge_kernel<OP, D, IO, UL, 1>;
+        if (int rc = ensure_smem(kernel, smem)) return rc;
+        kernel<<<pairs, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
+    }
     return finish_launch();
 }
 

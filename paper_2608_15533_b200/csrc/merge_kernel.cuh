@@ -1,4 +1,4 @@
-// Merge kernel: one CTA per (listed slot, head) folds the live log into the dense base with a
+// Merge kernel: a CTA folds the live log of a (listed slot, head) unit into its dense base with a
 // single read and a single write of the tile (Eq. 5 without the current-token term):
 //
 //   S_base[j, :] <- e^{lbar_j} S_base[j, :] + sum_{i<len} (e^{lbar_j - Lambda_ij} K_ij) U_i[:],   len <- 0
@@ -20,21 +20,53 @@ constexpr size_t merge_smem_bytes(int cap) {
 #ifndef DELTALOG_MERGE_CTAS
 #define DELTALOG_MERGE_CTAS 2
 #endif
-template <int OP, int D, typename IO, typename UL>
+// PACK: (listed slot, head) pairs a CTA is responsible for: 1 when every listed unit is expected to
+// fold, 8 for predicate merges over a batch with staggered fills, where most pairs are skipped.
+template <int OP, int D, typename IO, typename UL, int PACK>
 __global__ void __launch_bounds__(kThreads, DELTALOG_MERGE_CTAS)
-merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full) {
+merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
     constexpr bool kVecDecay = (OP != DELTALOG_GDN);
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL;
 
     const int tid = threadIdx.x;
-    const int n = blockIdx.x / st.H, h = blockIdx.x % st.H;
-    int slot;
-    if (!resolve_slot(slot_idx, n, st.num_slots, st.status, tid, slot)) return;
-    const size_t unit = (size_t)slot * st.H + h;
     const int cap = st.cap;
-    const int len = st.log_len[unit];
-    if (len <= 0 || len > cap || (only_if_full && len < cap)) return;  // nothing to fold: no dense write
+    // The lengths of a CTA's PACK candidates are looked up in parallel first, so a CTA whose
+    // candidates have nothing to fold costs one load latency, not PACK of them.
+    __shared__ int s_unit[PACK], s_len[PACK];
+    if (PACK > 1) {
+        if (tid < PACK) {
+            const int pair = blockIdx.x * PACK + tid;
+            int len = 0, unit = 0;
+            if (pair < n_pairs) {
+                int slot;
+                if (resolve_slot(slot_idx, pair / st.H, st.num_slots, st.status, 0, slot)) {
+                    unit = slot * st.H + pair % st.H;
+                    len = st.log_len[unit];
+                    if (len <= 0 || len > cap || (only_if_full && len < cap)) len = 0;  // nothing to fold
+                }
+            }
+            s_unit[tid] = unit;
+            s_len[tid] = len;
+        }
+        __syncthreads();
+    }
+    for (int cand = 0; cand < PACK; ++cand) {
+    int len;
+    size_t unit;
+    if (PACK > 1) {
+        len = s_len[cand];
+        if (len == 0) continue;
+        unit = (size_t)s_unit[cand];
+        if (cand > 0) __syncthreads();  // the previous candidate's shared-memory operands are no longer read
+    } else {
+        const int pair = blockIdx.x;
+        int slot;
+        if (!resolve_slot(slot_idx, pair / st.H, st.num_slots, st.status, tid, slot)) return;
+        unit = (size_t)slot * st.H + pair % st.H;
+        len = st.log_len[unit];
+        if (len <= 0 || len > cap || (only_if_full && len < cap)) return;  // nothing to fold: no dense write
+    }
 
     // each thread owns rows [rl*NP, rl*NP + NP) x columns [4*c4, 4*c4 + 4)
     float4 *Sg = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
@@ -93,6 +125,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full) {
 #pragma unroll
     for (int p = 0; p < NP; ++p) Sg[(size_t)(rl * NP + p) * C4 + c4] = s[p];
     if (tid == 0) st.log_len[unit] = 0;
+    }
 }
 
 }  // namespace deltalog
