@@ -102,6 +102,40 @@ def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float 
     return out
 
 
+def decode_merge_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float = 1.0) -> np.ndarray:
+    """One token through Algorithm 1's else-branch for every unit (whatever its live length):
+    readouts from the pre-update logical state, ``lbar += lambda_t``, factors (a, b), then Eq. 5 --
+    the represented state *plus the current update* is written into the base -- and the log is
+    cleared (``lbar = 0``, ``length = 0``).  Returns ``out [N, d_v]``."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    lam = np.asarray(lam, dtype=np.float64).reshape(st.N, st.d_lambda)
+    out = np.empty((st.N, st.d_v))
+    for n in range(st.N):
+        L = int(st.length[n])
+        # line 1: readouts defined on the pre-update logical state
+        S_prev = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L)
+        # line 2
+        st.lbar[n] = st.lbar[n] + lam[n]
+        S_decayed = _row_scale(lam[n], st.d_k)[:, None] * S_prev
+        # line 3
+        a = k[n]
+        if st.op == RWKV6:
+            b = v[n]
+            out[n] = S_prev.T @ q[n] + float(np.sum(q[n] * bonus[n] * k[n])) * v[n]
+        else:
+            b = float(beta[n]) * (v[n] - S_decayed.T @ k[n])
+        # lines 7-8 / Eq. 5: D(lbar) S_base + sum_i D(lbar - Lam[i]) K[i] U[i]^T + a b^T, then reset
+        S_new = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L) + np.outer(a, b)
+        if st.op != RWKV6:
+            out[n] = scale * (S_new.T @ q[n])
+        st.S_base[n] = S_new
+        st.lbar[n] = 0.0
+        st.length[n] = 0
+    return out
+
+
 def merge(st: LogState, only_if_full: bool = False) -> None:
     """Eq. 5 without the current-token term: fold the log into the base, reset lbar and length."""
     for n in range(st.N):

@@ -272,3 +272,29 @@ def test_log_schedule_merge_variants():
         logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t])
     with pytest.raises(RuntimeError):
         logical.decode_step(st, q[0], k[0], v[0], lam[0], beta=beta[0])
+
+
+@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+@pytest.mark.parametrize("cap", [1, 3, 4])
+def test_paper_cycle_with_fused_merge_step_equals_eager(op, cap):
+    """The paper's own cycle: cap appends, then one step that consumes a token AND materialises
+    (Algorithm 1, else-branch; Eq. 5 with the current-token term)."""
+    T, N, dk, dv = 13, 2, 4, 3
+    S0, q, k, v, lam, beta, bonus = rand_inputs(op, T, N, dk, dv)
+    ref = roll(op, S0, q, k, v, lam, beta, bonus, scale=0.9, snapshot_at=range(1, T + 1))
+    st = logical.LogState(op, S0, cap)
+    for t in range(T):
+        if (st.length == cap).all():
+            out = logical.decode_merge_step(st, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus, scale=0.9)
+            assert (st.length == 0).all() and (st.lbar == 0).all()
+            np.testing.assert_allclose(st.S_base, ref["snapshots"][t], atol=1e-12)   # base alone is the state
+        else:
+            out = logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus, scale=0.9)
+        np.testing.assert_allclose(out, ref["out"][t], atol=1e-12)
+        np.testing.assert_allclose(logical.materialize(st), ref["snapshots"][t], atol=1e-12)
+    # on an empty log the fused step is the eager step
+    st2 = logical.LogState(op, S0, cap)
+    for t in range(3):
+        out = logical.decode_merge_step(st2, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus, scale=0.9)
+        np.testing.assert_allclose(out, ref["out"][t], atol=1e-12)
+        np.testing.assert_allclose(st2.S_base, ref["snapshots"][t], atol=1e-12)
