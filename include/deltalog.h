@@ -103,6 +103,22 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
                          void *stream);
 
 /*
+ * The merge step of the cycle as the paper runs it (Algorithm 1, else-branch; Eq. 5 with the
+ * current-token term): every row of the batch consumes its token AND has its state materialised,
+ *     lbar <- lbar + lambda_t ;  (a_t, b_t) and `out` exactly as in deltalog_decode_step ;
+ *     S_base <- D(lbar) S_base + sum_i D(lbar - Lambda[i]) K[i] U[i]^T + a_t b_t^T ;  log_len <- 0
+ * whatever the live length of its log (0..cap; with an empty log this is the eager step on S_base).
+ * The token is NOT appended.  Arguments, layouts and status bits as for deltalog_decode_step;
+ * DELTALOG_STATUS_LOG_FULL is never raised.  The caller keeps phase-split batches (Section 4):
+ * rows whose log is full go through this call, the others through deltalog_decode_step.  One read
+ * and one write of each listed row's base tile.
+ */
+int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *state, const void *q,
+                               const void *k, const void *v, const float *g, const float *beta,
+                               const float *u_bonus, const int32_t *slot_idx, int32_t B, void *out,
+                               void *stream);
+
+/*
  * Materialise the log into the base (Eq. 5 without the current-token term):
  *     S_base <- D(lbar) S_base + sum_i D(lbar - Lambda[i]) K[i] U[i]^T ;  log_len <- 0
  * for the n slots listed in slot_idx (slots 0..n-1 if NULL), all heads.  A (slot, head) with an

@@ -9,6 +9,7 @@
 #include "decode_kernel.cuh"
 #include "decode_pipelined.cuh"
 #include "eager_kernel.cuh"
+#include "fused_step_kernel.cuh"
 #include "merge_kernel.cuh"
 
 namespace deltalog {
@@ -176,6 +177,16 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
 }
 
 template <int OP, int D, typename IO>
+int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
+    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    auto kernel = decode_merge_step_kernel<OP, D, IO, UL>;
+    const size_t smem = fused_step_smem_bytes<D>(st.cap);
+    if (int rc = ensure_smem(kernel, smem)) return rc;
+    kernel<<<tk.B * st.H, kThreads, smem, stream>>>(st, tk);
+    return finish_launch();
+}
+
+template <int OP, int D, typename IO>
 int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenArgs &tk, cudaStream_t stream) {
     eager_step_kernel<OP, D, IO><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
     return finish_launch();
@@ -221,6 +232,23 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
 #define CALL_DECODE(OP, D, IO) return launch_decode<OP, D, IO>(st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
 #undef CALL_DECODE
+    return DELTALOG_ERR_INVALID_ARG;
+}
+
+int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *state, const void *q,
+                               const void *k, const void *v, const float *g, const float *beta,
+                               const float *u_bonus, const int32_t *slot_idx, int32_t B, void *out,
+                               void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
+    if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
+    if (B == 0) return DELTALOG_OK;
+    const StateArgs st = make_state_args(desc, state);
+    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define CALL_FUSED(OP, D, IO) return launch_fused_step<OP, D, IO>(st, tk, s)
+    DELTALOG_DISPATCH(desc, CALL_FUSED);
+#undef CALL_FUSED
     return DELTALOG_ERR_INVALID_ARG;
 }
 

@@ -1,0 +1,178 @@
+// Fused merge step: one CTA per (batch row, head) consumes a token AND materialises the state
+// (Algorithm 1, else-branch; Eq. 5 with the current-token term a_t b_t^T), whatever the live length:
+//
+//   lbar  = Lambda[len-1] (0 if the log is empty),  lbar' = lbar + lambda_t
+//   delta ops:  S'  = D(lbar') S_base + sum_i D(lbar' - Lambda[i]) K[i] U[i]^T      (decayed state)
+//               b   = beta (v - S'^T k);  out = scale (S'^T q + (q.k) b);  S_base <- S' + k b^T
+//   RWKV6:      S-  = D(lbar) S_base + sum_i D(lbar - Lambda[i]) K[i] U[i]^T        (pre-update state)
+//               out = S-^T r + (r.(bonus.k)) v;                 S_base <- D(lambda_t) S- + k v^T
+//   len <- 0   (lbar is Lambda[len-1], so clearing the length clears it too)
+//
+// One read and one write of the tile, like the eager step, plus one read of the live log.  The tile
+// is requested first and held in registers: every thread owns NP consecutive rows x 4 columns.
+#pragma once
+
+#include "common.cuh"
+
+namespace deltalog {
+
+template <int D>
+__host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
+    constexpr int RL = kThreads / (D / 4);
+    // A [cap][D], U [cap][D], e, q, k, w, b [D] each, partial sums [RL][2][D], scalars
+    return sizeof(float) * ((size_t)2 * cap * D + 5 * D + 2 * D * RL + 4);
+}
+
+template <int OP, int D, typename IO, typename UL>
+__global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
+    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
+    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr int DL = kVecDecay ? D : 1;
+    constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL, EPL = D / 32;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    int slot;
+    if (!resolve_slot(tk.slot_idx, b, st.num_slots, st.status, tid, slot)) return;
+    const size_t unit = (size_t)slot * st.H + h, row = (size_t)b * st.H + h;
+    const int cap = st.cap;
+
+    float4 *Sg = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
+    const int c4 = tid % C4, rl = tid / C4;
+    float4 s[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) s[p] = Sg[(size_t)(rl * NP + p) * C4 + c4];
+
+    int len = st.log_len[unit];
+    len = len < 0 ? 0 : (len > cap ? cap : len);
+
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][D]  e^{lref_j - Lambda_ij} K_ij
+    float *U_s = A_s + (size_t)cap * D;                // [len][D]
+    float *e_s = U_s + (size_t)cap * D;                // e^{lref}
+    float *q_s = e_s + D;
+    float *k_s = q_s + D;
+    float *w_s = k_s + D;                              // RWKV6: e^{lambda_t}
+    float *b_s = w_s + D;
+    float *red_s = b_s + D;                            // [RL][2][D]
+    float *scal_s = red_s + 2 * D * RL;                // [0] = q.k  (or r.(bonus.k))
+
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const float *Lg = st.decay_log + unit * cap * DL;
+    const float *lold = Lg + (size_t)(len > 0 ? len - 1 : 0) * DL;
+    const float *gg = tk.g + row * DL;
+    // lref: the decay level the state is materialised at -- lbar' for the delta rule (both readouts
+    // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
+    if (!kVecDecay) {
+        const float lref = (len > 0 ? lold[0] : 0.f) + gg[0];
+        for (int x = tid * 4; x < len * D; x += kThreads * 4) {
+            const float wi = expf(lref - Lg[x / D]);
+            float kv[4], uv[4];
+            load_vec<IO, 4>(Kg + x, kv);
+            load_vec<UL, 4>(Ug + x, uv);
+            *reinterpret_cast<float4 *>(A_s + x) = make_float4(wi * kv[0], wi * kv[1], wi * kv[2], wi * kv[3]);
+            *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
+        }
+    } else {
+        for (int x = tid; x < len * D; x += kThreads) {
+            const int i = x / D, j = x % D;
+            const float lref = lold[j] + (kDelta ? gg[j] : 0.f);
+            A_s[x] = expf(lref - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);
+            U_s[x] = to_f32(Ug[x]);
+        }
+    }
+    const IO *vg = static_cast<const IO *>(tk.v) + row * D;
+    if (tid < D) {
+        const int jl = kVecDecay ? tid : 0;
+        const float lo = len > 0 ? lold[jl] : 0.f, lam = gg[jl];
+        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[row * D + tid]);
+        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[row * D + tid]);
+        e_s[tid] = expf(kDelta ? lo + lam : lo);
+        w_s[tid] = expf(lam);
+    }
+    __syncthreads();
+
+    if (warp == 0) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
+        float d = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const int j = lane + 32 * e;
+            const float w = kDelta ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            d = fmaf(q_s[j] * w, k_s[j], d);
+        }
+        d = warp_sum(d);
+        if (lane == 0) scal_s[0] = d;
+    }
+
+    // materialise at lref (Eq. 6) in registers
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const float e = e_s[rl * NP + p];
+        s[p] = make_float4(e * s[p].x, e * s[p].y, e * s[p].z, e * s[p].w);
+    }
+    const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
+    for (int i = 0; i < len; ++i) {
+        const float4 u = U4[i * C4 + c4];
+        const float4 *a4 = reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP);
+#pragma unroll
+        for (int p4 = 0; p4 < NP / 4; ++p4) {
+            const float4 a = a4[p4];
+            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
+            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
+            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
+            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
+        }
+    }
+
+    // the two readouts from the materialised tile
+    float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), aq = ak;
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int r = rl * NP + p;
+        if (kDelta) ak = fma4(k_s[r], s[p], ak);
+        aq = fma4(q_s[r], s[p], aq);
+    }
+    float4 *red4 = reinterpret_cast<float4 *>(red_s);
+    if (kDelta) red4[(rl * 2 + 0) * C4 + c4] = ak;
+    red4[(rl * 2 + 1) * C4 + c4] = aq;
+    __syncthreads();
+
+    const int which = tid / D, c = tid % D;  // which: 0 -> S'^T k half, 1 -> S'^T q half
+    const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+    const int sel = kDelta ? which : 1;
+    float y = 0.f;
+    if (active) {
+#pragma unroll
+        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+    }
+    IO *og = static_cast<IO *>(tk.out) + row * D;
+    if (kDelta) {
+        if (tid < D) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
+        __syncthreads();
+        if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
+    } else {
+        if (active) {
+            const float vv = to_f32(vg[c]);
+            b_s[c] = vv;
+            og[c] = from_f32<IO>(fmaf(scal_s[0], vv, y));
+        }
+        __syncthreads();
+    }
+
+    // Eq. 5: the represented state plus the current update, written once; the log is cleared
+    const float4 b4 = reinterpret_cast<const float4 *>(b_s)[c4];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int r = rl * NP + p;
+        float4 x = s[p];
+        if (!kDelta) {
+            const float a = w_s[r];
+            x = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
+        }
+        Sg[(size_t)r * C4 + c4] = fma4(k_s[r], b4, x);
+    }
+    if (tid == 0) st.log_len[unit] = 0;
+}
+
+}  // namespace deltalog

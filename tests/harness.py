@@ -112,9 +112,13 @@ def oracle_for(wl: Workload, rec: Recorded, S0_units: np.ndarray, bonus_units: O
 def run_deltalog(wl: Workload, cap: int, device, *, units: Sequence[Tuple[int, int]], scale: float = 1.0,
                  slot_idx: Optional[torch.Tensor] = None, start_delay: Optional[torch.Tensor] = None,
                  generator_device: str = "cpu", steps: Optional[int] = None, final_merge: bool = True,
-                 every_step_hook=None):
+                 every_step_hook=None, cycle: str = "split"):
     """Decode ``steps`` tokens with the log schedule: merge (only full logs) before every step, one
     call over the whole batch, which is the launch configuration the benchmark times.
+
+    ``cycle="paper"`` runs the paper's own cycle instead (Algorithm 1): no token-less merge; rows
+    whose log is full take the fused merge step, the others append -- two calls over phase-split
+    batches (a row sits out of a call with slot index -1).
 
     ``start_delay``: optional int ``[batch]``; row b sits out (slot index -1) until global step
     ``start_delay[b]``, so merge boundaries are staggered across the batch by real decode steps
@@ -145,13 +149,24 @@ def run_deltalog(wl: Workload, cap: int, device, *, units: Sequence[Tuple[int, i
         step_slots = sidx
         if delay is not None:
             step_slots = torch.where(delay <= t, all_slots, torch.full_like(all_slots, -1))
-        dl.merge(desc, state, slot_idx=sidx, n=wl.batch, only_if_full=True)
+        if cycle == "split":
+            dl.merge(desc, state, slot_idx=sidx, n=wl.batch, only_if_full=True)
         if delay is None and t > 0 and bool((state.log_len[uslot, uh] == 0).all()):
             rec.state_at.append(t)
             rec.states.append(f64(state.S_base[uslot, uh]))
         tok = {k_: (v_.to(device) if v_ is not None else None) for k_, v_ in src.token().items()}
-        out = dl.decode_step(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
-                             u_bonus=bonus, slot_idx=step_slots)
+        if cycle == "split":
+            out = dl.decode_step(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                                 u_bonus=bonus, slot_idx=step_slots)
+        else:
+            rows = step_slots if step_slots is not None else all_slots
+            full = state.log_len[all_slots.long(), 0] == cap  # heads of a row fill in lockstep
+            skip = torch.full_like(all_slots, -1)
+            out = torch.zeros(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
+            for fn, sel in ((dl.decode_step, ~full), (dl.decode_merge_step, full)):
+                if bool(sel.any()):
+                    fn(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,
+                       slot_idx=torch.where(sel, rows, skip), out=out)
         rec.record_token(tok, out, wl)
         if every_step_hook is not None:
             every_step_hook(t, state, tok, out)
