@@ -141,6 +141,11 @@ class Rig:
                             beta=tok["beta"], u_bonus=self.bonus[layer],
                             slot_idx=self.slot_idx if slot_idx is None else slot_idx, out=self.out)
 
+    def fused(self, t, layer=0):
+        tok = self.rings[layer][t % self.RING]
+        self.dl.decode_merge_step(self.desc, self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
+                                  beta=tok["beta"], u_bonus=self.bonus[layer], slot_idx=self.slot_idx, out=self.out)
+
     def merge(self, layer=0, only_if_full=None):
         if only_if_full is None:   # a uniform batch folds every row at once; a staggered one uses the predicate
             only_if_full = self.staggered
@@ -260,6 +265,79 @@ def time_graph_loop(rig: Rig, steps: int):
     torch.cuda.synchronize()
     launch.barrier()
     return start.elapsed_time(end)
+
+
+def time_paper_cycle(rig: Rig, steps: int):
+    """The paper's own cycle (Algorithm 1): cap appends, then one fused step that consumes a token and
+    materialises; cap + 1 tokens per dense write.  Uniform batch: one launch per step.  Staggered batch
+    (fills uniform on 0..cap): every step is two launches over phase-split batches -- the append
+    call sees slot -1 for the rows whose log is full, the fused-step call for all the others; the
+    host knows each row's phase from its step counter, so the lists are precomputed for one period.
+    Timed as CUDA-graph replays of whole cycles; on a single-layer uniform batch the fused step alone
+    is then timed over plain launches with one event pair per cycle.
+    Returns (steps timed, total ms, mean ms of a fused-step launch or None)."""
+    import math
+
+    cap, M = rig.cap, rig.cap + 1
+    g_len = M * Rig.RING // math.gcd(M, Rig.RING)
+    steps = max(steps // g_len, 1) * g_len
+    for layer in range(rig.layers):
+        rig.merge(layer, only_if_full=False)
+    dl = rig.dl
+    app_lists = mrg_lists = None
+    if rig.staggered:
+        delay = workloads.fill_offsets(rig.wl, M).to(rig.device)   # row b starts `delay` steps late: fill cap - delay
+        skip = torch.full_like(rig.slot_idx, -1)
+        for t in range(cap):
+            slots = torch.where(delay <= t, rig.slot_idx, skip)
+            for layer in range(rig.layers):
+                rig.decode(t, layer, slot_idx=slots)
+        full_at = [((tau - delay) % M) == 0 for tau in range(M)]     # row is full before step tau of a period
+        app_lists = [torch.where(f, skip, rig.slot_idx) for f in full_at]
+        mrg_lists = [torch.where(f, rig.slot_idx, skip) for f in full_at]
+
+    def one(t, layer):
+        tok = rig.rings[layer][t % rig.RING]
+        args = (rig.desc, rig.states[layer], tok["q"], tok["k"], tok["v"], tok["g"])
+        kw = dict(beta=tok["beta"], u_bonus=rig.bonus[layer], out=rig.out)
+        if rig.staggered:
+            dl.decode_step(*args, slot_idx=app_lists[t % M], **kw)
+            dl.decode_merge_step(*args, slot_idx=mrg_lists[t % M], **kw)
+        else:
+            (dl.decode_merge_step if t % M == M - 1 else dl.decode_step)(*args, slot_idx=rig.slot_idx, **kw)
+
+    stream = torch.cuda.Stream(device=rig.device)
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            for t in range(g_len):
+                for layer in range(rig.layers):
+                    one(t, layer)
+        graph.replay()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(stream):
+        start.record()
+        for _ in range(steps // g_len):
+            graph.replay()
+        end.record()
+    torch.cuda.synchronize()
+    total = start.elapsed_time(end)
+    fused_ms = None
+    if not rig.staggered and rig.layers == 1:
+        marks = []
+        for t in range(min(steps, 32 * M)):
+            if t % M == M - 1:
+                marks.append((torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)))
+                marks[-1][0].record()
+                one(t, 0)
+                marks[-1][1].record()
+            else:
+                one(t, 0)
+        torch.cuda.synchronize()
+        fused_ms = statistics.mean(a.elapsed_time(b) for a, b in marks)
+    return steps, total, fused_ms
 
 
 def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = True):
@@ -513,6 +591,21 @@ def main():
                                 "hbm_gbs": eager_bytes / (eager_ms * 1e-3) / 1e9,
                                 "bytes_written_per_unit_step": traffic.eager_write(u)}
         line["speedup_vs_eager_kernel"] = eager_ms / (ms_per_step / layers)
+        # the paper's own cycle: cap appends + one fused merge step (cap + 1 tokens per dense write)
+        p_steps, p_ms, fused_ms = time_paper_cycle(rig, args.steps)
+        pc = traffic.paper_cycle_bytes(u, cap + 1)
+        p_step_ms = p_ms / p_steps
+        line["paper_cycle"] = {
+            "ms_per_step": p_step_ms, "value": units * layers * p_steps / (p_ms * 1e-3), "steps": p_steps,
+            "merge_interval_M": cap + 1, "algorithmic_bytes_per_unit_step": pc["total"],
+            "hbm_gbs": pc["total"] * units * layers / (p_step_ms * 1e-3) / 1e9,
+            "launch": ("two launches per layer-step over phase-split batches" if stag else "one launch per step"),
+            "speedup_vs_eager_kernel": eager_ms / (p_step_ms / layers)}
+        if fused_ms is not None:
+            fused_bytes = (traffic.fused_read(u, cap) + traffic.fused_write(u)) * units
+            line["paper_cycle"]["fused_step_ms"] = fused_ms
+            line["paper_cycle"]["fused_step_hbm_gbs"] = fused_bytes / (fused_ms * 1e-3) / 1e9
+        assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
         sweep = {}
         for c in wl.caps:
             if c == cap and layers == 1:

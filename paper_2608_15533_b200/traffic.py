@@ -73,6 +73,16 @@ def merge_write(u: UnitShape) -> int:
     return u.state + LEN_WORD
 
 
+def fused_read(u: UnitShape, fill: int) -> int:
+    """Bytes the fused merge step reads with ``fill`` live entries: base + live log + token + length."""
+    return u.state + fill * u.entry + u.token_in + LEN_WORD
+
+
+def fused_write(u: UnitShape) -> int:
+    """Bytes the fused merge step writes: the base, the output, the length."""
+    return u.state + u.token_out + LEN_WORD
+
+
 def eager_read(u: UnitShape) -> int:
     return u.state + u.token_in
 
