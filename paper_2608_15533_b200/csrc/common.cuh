@@ -81,6 +81,64 @@ __device__ __forceinline__ float4 fma4(float a, const float4 &x, const float4 &a
     return make_float4(fmaf(a, x.x, acc.x), fmaf(a, x.y, acc.y), fmaf(a, x.z, acc.z), fmaf(a, x.w, acc.w));
 }
 
+// Rank-len update of a thread's NP consecutive rows x 4 columns held in registers:
+//     s[p] += sum_{i<len} A_i[p] * u_i,   load_a(i, p4) -> A_i for rows 4*p4 .. 4*p4+3,  load_u(i) -> u_i.
+// The accumulators are kept as pairs of rows so that one packed fp32 FMA (two lanes per instruction)
+// serves two rows: per entry 4 register packs and NP*2 packed FMAs instead of NP*4 scalar ones.
+// Every element sees the same fused multiply-adds in the same order as the scalar form.
+#ifndef DELTALOG_FFMA2
+#define DELTALOG_FFMA2 1
+#endif
+template <int NP, typename LoadA, typename LoadU>
+__device__ __forceinline__ void rank_update(float4 (&s)[NP], int len, LoadA load_a, LoadU load_u) {
+    static_assert(NP % 4 == 0, "rows come in groups of four");
+#if DELTALOG_FFMA2
+    float2 acc[NP / 2][4];
+#pragma unroll
+    for (int pp = 0; pp < NP / 2; ++pp) {
+        acc[pp][0] = make_float2(s[2 * pp].x, s[2 * pp + 1].x);
+        acc[pp][1] = make_float2(s[2 * pp].y, s[2 * pp + 1].y);
+        acc[pp][2] = make_float2(s[2 * pp].z, s[2 * pp + 1].z);
+        acc[pp][3] = make_float2(s[2 * pp].w, s[2 * pp + 1].w);
+    }
+    for (int i = 0; i < len; ++i) {
+        const float4 u = load_u(i);
+        const float2 u0 = make_float2(u.x, u.x), u1 = make_float2(u.y, u.y);
+        const float2 u2 = make_float2(u.z, u.z), u3 = make_float2(u.w, u.w);
+#pragma unroll
+        for (int p4 = 0; p4 < NP / 4; ++p4) {
+            const float4 a = load_a(i, p4);
+            const float2 a01 = make_float2(a.x, a.y), a23 = make_float2(a.z, a.w);
+            acc[2 * p4][0] = __ffma2_rn(a01, u0, acc[2 * p4][0]);
+            acc[2 * p4][1] = __ffma2_rn(a01, u1, acc[2 * p4][1]);
+            acc[2 * p4][2] = __ffma2_rn(a01, u2, acc[2 * p4][2]);
+            acc[2 * p4][3] = __ffma2_rn(a01, u3, acc[2 * p4][3]);
+            acc[2 * p4 + 1][0] = __ffma2_rn(a23, u0, acc[2 * p4 + 1][0]);
+            acc[2 * p4 + 1][1] = __ffma2_rn(a23, u1, acc[2 * p4 + 1][1]);
+            acc[2 * p4 + 1][2] = __ffma2_rn(a23, u2, acc[2 * p4 + 1][2]);
+            acc[2 * p4 + 1][3] = __ffma2_rn(a23, u3, acc[2 * p4 + 1][3]);
+        }
+    }
+#pragma unroll
+    for (int pp = 0; pp < NP / 2; ++pp) {
+        s[2 * pp] = make_float4(acc[pp][0].x, acc[pp][1].x, acc[pp][2].x, acc[pp][3].x);
+        s[2 * pp + 1] = make_float4(acc[pp][0].y, acc[pp][1].y, acc[pp][2].y, acc[pp][3].y);
+    }
+#else
+    for (int i = 0; i < len; ++i) {
+        const float4 u = load_u(i);
+#pragma unroll
+        for (int p4 = 0; p4 < NP / 4; ++p4) {
+            const float4 a = load_a(i, p4);
+            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
+            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
+            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
+            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
+        }
+    }
+#endif
+}
+
 // Resolve the pool slot of batch row b; returns false when the row must be skipped.
 __device__ __forceinline__ bool resolve_slot(const int32_t *slot_idx, int b, int num_slots, int32_t *status,
                                              int tid, int &slot) {

@@ -112,18 +112,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
         s[p] = make_float4(e * s[p].x, e * s[p].y, e * s[p].z, e * s[p].w);
     }
     const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
-    for (int i = 0; i < len; ++i) {
-        const float4 u = U4[i * C4 + c4];
-        const float4 *a4 = reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP);
-#pragma unroll
-        for (int p4 = 0; p4 < NP / 4; ++p4) {
-            const float4 a = a4[p4];
-            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
-            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
-            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
-            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
-        }
-    }
+    rank_update<NP>(
+        s, len,
+        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP)[p4]; },
+        [&](int i) { return U4[i * C4 + c4]; });
 
     // the two readouts from the materialised tile
     float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), aq = ak;

@@ -110,18 +110,10 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
         s[p] = make_float4(e * s[p].x, e * s[p].y, e * s[p].z, e * s[p].w);
     }
     const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
-    for (int i = 0; i < len; ++i) {
-        const float4 u = U4[i * C4 + c4];
-        const float4 *a4 = reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP);
-#pragma unroll
-        for (int p4 = 0; p4 < NP / 4; ++p4) {
-            const float4 a = a4[p4];
-            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
-            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
-            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
-            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
-        }
-    }
+    rank_update<NP>(
+        s, len,
+        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP)[p4]; },
+        [&](int i) { return U4[i * C4 + c4]; });
 #pragma unroll
     for (int p = 0; p < NP; ++p) Sg[(size_t)(rl * NP + p) * C4 + c4] = s[p];
     if (tid == 0) st.log_len[unit] = 0;
