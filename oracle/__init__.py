@@ -6,7 +6,8 @@ imports nothing from it.
 
 Contents
 --------
-``eager_rollout``      the eager dense recurrence of GDN / KDA / RWKV6 (Eq. 3, Table 1), compiled
+``eager_rollout``      the eager dense recurrence of GDN / KDA / RWKV6 and of the additive family
+                       (linear attention, RetNet, GLA) (Eq. 3, Table 1), compiled
                        from ``eager_oracle.c`` (plain C, fp64, OpenMP over independent units).
 ``logical``            the base-plus-log schedule of Algorithm 1 / Eq. 4-6 in fp64 numpy, used to
                        check the physical state (base, log, snapshots) that the GPU leaves behind.
@@ -25,8 +26,8 @@ import numpy as np
 
 from . import logical  # noqa: F401  (re-export)
 
-GDN, KDA, RWKV6 = 0, 1, 2
-OP_BY_NAME = {"gdn": GDN, "kda": KDA, "rwkv6": RWKV6}
+GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+OP_BY_NAME = {"gdn": GDN, "kda": KDA, "rwkv6": RWKV6, "linattn": LINATTN, "retnet": RETNET, "gla": GLA}
 
 _HERE = Path(__file__).resolve().parent
 _SRC = _HERE / "eager_oracle.c"
@@ -83,8 +84,8 @@ def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapsh
     """Eager fp64 recurrence over ``T`` tokens for ``N`` independent (sequence, head) units.
 
     Shapes: ``S0 [N,d_k,d_v]``, ``q,k [T,N,d_k]``, ``v [T,N,d_v]``, ``lam [T,N,d_lambda]`` (log-decay;
-    ``d_lambda`` = 1 for GDN, ``d_k`` for KDA / RWKV6), ``beta [T,N]`` (GDN / KDA),
-    ``bonus [N,d_k]`` (RWKV6).  ``snapshot_at``: ascending 1-based token counts.
+    ``d_lambda`` = 1 for GDN / RetNet, ``d_k`` for KDA / RWKV6 / GLA; ignored for plain linear
+    attention), ``beta [T,N]`` (GDN / KDA), ``bonus [N,d_k]`` (RWKV6).  ``snapshot_at``: ascending 1-based token counts.
 
     Returns ``dict(out [T,N,d_v], b [T,N,d_v], S [N,d_k,d_v], snapshots [n,N,d_k,d_v])``;
     ``b`` is the value-side factor of every token (what the log's U entries must hold).
@@ -94,7 +95,9 @@ def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapsh
     S0 = np.asarray(S0, dtype=np.float64)
     N, d_k, d_v = S0.shape
     T = int(np.asarray(q).shape[0])
-    d_lambda = 1 if op == GDN else d_k
+    d_lambda = 1 if op in (GDN, RETNET, LINATTN) else d_k
+    if op == LINATTN:
+        lam = np.zeros((T, N, 1))  # no decay: the C side does not read it
     S = np.array(S0, dtype=np.float64, order="C", copy=True)
     q = _f64(q, (T, N, d_k))
     k = _f64(k, (T, N, d_k))
@@ -105,6 +108,8 @@ def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapsh
             raise ValueError("RWKV6 needs the bonus vector")
         bonus = _f64(bonus, (N, d_k))
         beta = None
+    elif op in (LINATTN, RETNET, GLA):
+        beta = bonus = None
     else:
         if beta is None:
             raise ValueError("GDN / KDA need beta")

@@ -1,8 +1,9 @@
 /*
  * TEST INFRASTRUCTURE -- the parity oracle. Not part of the product path.
  *
- * Plain fp64 eager recurrence for the three recurrent linear-attention
- * operators whose decode update this repository accelerates (GDN, KDA, RWKV6).
+ * Plain fp64 eager recurrence for the recurrent linear-attention operators whose
+ * decode update this repository accelerates (GDN, KDA, RWKV6 and the additive
+ * family of Table 1: plain linear attention, RetNet, GLA).
  * "Eager" means the dense d_k x d_v state is rewritten at every token, which is
  * the definition the deferred (base + log) schedule must reproduce exactly in
  * exact arithmetic (Section 3, Eq. 6 and the closure argument below it).
@@ -17,6 +18,9 @@
  *   KDA   per-key lambda, same a, b, o
  *   RWKV6 per-key lambda (log w), a = k, b = v,
  *         o = S_{t-1}^T r + (r . (bonus (.) k)) v       (readout from the pre-update state)
+ *   Linear attention  no decay,         a = k (the caller applies the feature map), b = v
+ *   RetNet            scalar lambda,    a = k, b = v
+ *   GLA               per-key lambda,   a = k, b = v;   all three: o = scale * S_t^T q  (Eq. 3)
  *
  * Reading taken where the paper's Table 1 is ambiguous: the delta-rule
  * correction k^T S_{t-1} is evaluated on the *decayed* previous state, as the
@@ -37,7 +41,7 @@
 #include <omp.h>
 #endif
 
-enum { ORACLE_GDN = 0, ORACLE_KDA = 1, ORACLE_RWKV6 = 2 };
+enum { ORACLE_GDN = 0, ORACLE_KDA = 1, ORACLE_RWKV6 = 2, ORACLE_LINATTN = 3, ORACLE_RETNET = 4, ORACLE_GLA = 5 };
 
 /* One token of the gated delta rule (GDN: d_lambda == 1, KDA: d_lambda == d_k). */
 static void delta_rule_token(int d_k, int d_v, int d_lambda, double scale, double *S,
@@ -64,6 +68,24 @@ static void delta_rule_token(int d_k, int d_v, int d_lambda, double scale, doubl
         double acc = 0.0;
         for (j = 0; j < d_k; ++j) acc += S[(size_t)j * d_v + c] * q[j];
         o[c] = scale * acc;
+    }
+}
+
+/* One token of the additive family (Table 1: linear attention d_lambda == 0, RetNet d_lambda == 1,
+ * GLA d_lambda == d_k): S_t = D(lambda_t) S_{t-1} + k_t v_t^T, o_t = scale * S_t^T q_t   (Eq. 3). */
+static void additive_token(int d_k, int d_v, int d_lambda, double scale, double *S, const double *q,
+                           const double *k, const double *v, const double *lambda, double *o, double *b)
+{
+    int j, c;
+    for (j = 0; j < d_k; ++j) {
+        double a = d_lambda == 0 ? 1.0 : exp(lambda[d_lambda == 1 ? 0 : j]);
+        for (c = 0; c < d_v; ++c) S[(size_t)j * d_v + c] = a * S[(size_t)j * d_v + c] + k[j] * v[c];
+    }
+    for (c = 0; c < d_v; ++c) {
+        double acc = 0.0;
+        for (j = 0; j < d_k; ++j) acc += S[(size_t)j * d_v + c] * q[j];
+        o[c] = scale * acc;
+        b[c] = v[c];
     }
 }
 
@@ -96,7 +118,8 @@ static void rwkv6_token(int d_k, int d_v, double *S, const double *r, const doub
  *   S        [N][d_k][d_v]   in: S_0, out: S_T (updated in place)
  *   q, k     [T][N][d_k]     (q is r for RWKV6)
  *   v        [T][N][d_v]
- *   lambda   [T][N][d_lambda] log-decay, d_lambda = 1 (GDN) or d_k (KDA, RWKV6)
+ *   lambda   [T][N][d_lambda] log-decay, d_lambda = 1 (GDN, RetNet) or d_k (KDA, RWKV6, GLA);
+ *                            ignored (may be NULL) for plain linear attention
  *   beta     [T][N]          GDN / KDA only (may be NULL for RWKV6)
  *   bonus    [N][d_k]        RWKV6 only (may be NULL otherwise)
  *   out      [T][N][d_v]
@@ -112,9 +135,9 @@ int oracle_eager_rollout(int op, int T, int N, int d_k, int d_v, double scale, d
                          const double *beta, const double *bonus, double *out, double *b_rec,
                          int n_snap, const int *snap_at, double *S_snap)
 {
-    int d_lambda = (op == ORACLE_GDN) ? 1 : d_k;
+    int d_lambda = (op == ORACLE_GDN || op == ORACLE_RETNET) ? 1 : (op == ORACLE_LINATTN ? 0 : d_k);
     int n;
-    if (op != ORACLE_GDN && op != ORACLE_KDA && op != ORACLE_RWKV6) return -1;
+    if (op < ORACLE_GDN || op > ORACLE_GLA) return -1;
 #pragma omp parallel for schedule(dynamic, 1)
     for (n = 0; n < N; ++n) {
         double *Sn = S + (size_t)n * d_k * d_v;
@@ -127,6 +150,9 @@ int oracle_eager_rollout(int op, int T, int N, int d_k, int d_v, double scale, d
             if (op == ORACLE_RWKV6)
                 rwkv6_token(d_k, d_v, Sn, q + tn * d_k, k + tn * d_k, v + tn * d_v,
                             lambda + tn * d_lambda, bonus + (size_t)n * d_k, o, b);
+            else if (op >= ORACLE_LINATTN)
+                additive_token(d_k, d_v, d_lambda, scale, Sn, q + tn * d_k, k + tn * d_k, v + tn * d_v,
+                               d_lambda ? lambda + tn * d_lambda : NULL, o, b);
             else
                 delta_rule_token(d_k, d_v, d_lambda, scale, Sn, q + tn * d_k, k + tn * d_k,
                                  v + tn * d_v, lambda + tn * d_lambda, beta[tn], o, b);

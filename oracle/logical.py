@@ -20,7 +20,8 @@ from __future__ import annotations
 
 import numpy as np
 
-GDN, KDA, RWKV6 = 0, 1, 2
+GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+ADDITIVE = (LINATTN, RETNET, GLA)  # b = v, readout from the updated state; LINATTN: lambda == 0
 
 
 class LogState:
@@ -31,7 +32,7 @@ class LogState:
         self.op = int(op)
         self.N, self.d_k, self.d_v = S0.shape
         self.cap = int(cap)
-        self.d_lambda = 1 if self.op == GDN else self.d_k
+        self.d_lambda = 1 if self.op in (GDN, RETNET, LINATTN) else self.d_k
         self.S_base = S0.copy()
         self.lbar = np.zeros((self.N, self.d_lambda))
         self.K_log = np.zeros((self.N, self.cap, self.d_k))
@@ -64,6 +65,13 @@ def materialize(st: LogState) -> np.ndarray:
     ])
 
 
+def _lam(st: LogState, lam) -> np.ndarray:
+    """The token's log-decay as [N, d_lambda]; plain linear attention has none (zeros)."""
+    if st.op == LINATTN:
+        return np.zeros((st.N, st.d_lambda))
+    return np.asarray(lam, dtype=np.float64).reshape(st.N, st.d_lambda)
+
+
 def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float = 1.0) -> np.ndarray:
     """One token through Algorithm 1's append branch for every unit; returns ``out [N, d_v]``.
 
@@ -73,7 +81,7 @@ def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float 
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
-    lam = np.asarray(lam, dtype=np.float64).reshape(st.N, st.d_lambda)
+    lam = _lam(st, lam)
     out = np.empty((st.N, st.d_v))
     for n in range(st.N):
         L = int(st.length[n])
@@ -89,6 +97,8 @@ def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float 
         if st.op == RWKV6:
             b = v[n]
             out[n] = S_prev.T @ q[n] + float(np.sum(q[n] * bonus[n] * k[n])) * v[n]
+        elif st.op in ADDITIVE:
+            b = v[n]
         else:
             b = float(beta[n]) * (v[n] - S_decayed.T @ k[n])
         # lines 4-5 / Eq. 4: append (a, b, lbar) into slot L; the base is untouched
@@ -110,7 +120,7 @@ def decode_merge_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: 
     q = np.asarray(q, dtype=np.float64)
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
-    lam = np.asarray(lam, dtype=np.float64).reshape(st.N, st.d_lambda)
+    lam = _lam(st, lam)
     out = np.empty((st.N, st.d_v))
     for n in range(st.N):
         L = int(st.length[n])
@@ -124,6 +134,8 @@ def decode_merge_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: 
         if st.op == RWKV6:
             b = v[n]
             out[n] = S_prev.T @ q[n] + float(np.sum(q[n] * bonus[n] * k[n])) * v[n]
+        elif st.op in ADDITIVE:
+            b = v[n]
         else:
             b = float(beta[n]) * (v[n] - S_decayed.T @ k[n])
         # lines 7-8 / Eq. 5: D(lbar) S_base + sum_i D(lbar - Lam[i]) K[i] U[i]^T + a b^T, then reset

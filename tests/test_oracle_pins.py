@@ -14,14 +14,16 @@ import numpy as np
 import pytest
 
 import oracle
-from oracle import GDN, KDA, RWKV6, logical
+from oracle import GDN, GLA, KDA, LINATTN, RETNET, RWKV6, logical
+
+ALL_OPS = [GDN, KDA, RWKV6, LINATTN, RETNET, GLA]
 
 RNG = np.random.default_rng(12345)
 
 
 def rand_inputs(op, T, N, dk, dv, rng=None, unit_keys=False):
     rng = rng or np.random.default_rng(T * 1000 + N * 100 + dk * 10 + dv + op)
-    dl = 1 if op == GDN else dk
+    dl = 1 if op in (GDN, RETNET, LINATTN) else dk
     S0 = rng.normal(0, 0.3, (N, dk, dv))
     q = rng.normal(0, 1, (T, N, dk))
     k = rng.normal(0, 1, (T, N, dk))
@@ -29,6 +31,8 @@ def rand_inputs(op, T, N, dk, dv, rng=None, unit_keys=False):
         k /= np.linalg.norm(k, axis=-1, keepdims=True)
     v = rng.normal(0, 1, (T, N, dv))
     lam = -np.log1p(np.exp(rng.normal(0, 1, (T, N, dl))))
+    if op == LINATTN:
+        lam = np.zeros((T, N, 1))   # plain linear attention has no decay
     beta = 1 / (1 + np.exp(-rng.normal(0, 1, (T, N))))
     bonus = rng.normal(0, 0.5, (N, dk))
     return S0, q, k, v, lam, beta, bonus
@@ -37,6 +41,8 @@ def rand_inputs(op, T, N, dk, dv, rng=None, unit_keys=False):
 def roll(op, S0, q, k, v, lam, beta, bonus, **kw):
     if op == RWKV6:
         return oracle.eager_rollout(op, S0, q, k, v, lam, bonus=bonus, **kw)
+    if op in (LINATTN, RETNET, GLA):
+        return oracle.eager_rollout(op, S0, q, k, v, lam, **kw)
     return oracle.eager_rollout(op, S0, q, k, v, lam, beta=beta, **kw)
 
 
@@ -222,9 +228,57 @@ def test_oracle_rejects_bad_arguments():
 
 
 # ---------------------------------------------------------------------------------------------
+# additive family (Table 1: linear attention, RetNet, GLA): the parallel (attention-matrix) form
+# ---------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("op", [LINATTN, RETNET, GLA])
+@pytest.mark.parametrize("T,dk,dv", [(1, 2, 3), (6, 4, 3), (9, 3, 5)])
+def test_additive_family_matches_decay_masked_attention(op, T, dk, dv):
+    """o_t = scale * [ (q_t . e^{L_t})^T S_0 + sum_{s<=t} ((q_t . e^{L_t - L_s}) . k_s) v_s ] with L the
+    running sum of the log-decays (zero for linear attention, one scalar per head for RetNet): the
+    masked-attention form these models are trained in; S_T likewise as a sum of decayed outer products."""
+    N, scale = 2, 0.8
+    S0, q, k, v, lam, _, _ = rand_inputs(op, T, N, dk, dv)
+    res = roll(op, S0, q, k, v, lam, None, None, scale=scale)
+    lam_full = np.broadcast_to(lam, (T, N, dk)) if lam.shape[-1] == 1 else lam
+    Lc = np.cumsum(lam_full, axis=0)                                   # [T, N, dk]
+    for n in range(N):
+        for t in range(T):
+            o = (q[t, n] * np.exp(Lc[t, n])) @ S0[n]
+            for s_ in range(t + 1):
+                o = o + np.dot(q[t, n] * np.exp(Lc[t, n] - Lc[s_, n]), k[s_, n]) * v[s_, n]
+            np.testing.assert_allclose(res["out"][t, n], scale * o, atol=1e-12)
+        S_T = np.exp(Lc[T - 1, n])[:, None] * S0[n]
+        for s_ in range(T):
+            S_T = S_T + np.outer(np.exp(Lc[T - 1, n] - Lc[s_, n]) * k[s_, n], v[s_, n])
+        np.testing.assert_allclose(res["S"][n], S_T, atol=1e-12)
+    np.testing.assert_array_equal(res["b"], v)
+
+
+def test_additive_family_reductions():
+    """GLA with equal channels is RetNet; RetNet with gamma = 1 is linear attention; linear attention
+    from a zero state is the causal prefix sum of Eq. 1; RWKV6 with w = 1 and u = 1 reads the same
+    state one token later."""
+    T, N, dk, dv = 7, 2, 4, 3
+    S0, q, k, v, lam1, _, _ = rand_inputs(RETNET, T, N, dk, dv)
+    ret = oracle.eager_rollout(RETNET, S0, q, k, v, lam1, scale=1.1)
+    gla = oracle.eager_rollout(GLA, S0, q, k, v, np.repeat(lam1, dk, axis=-1), scale=1.1)
+    np.testing.assert_allclose(gla["out"], ret["out"], atol=1e-13)
+    np.testing.assert_allclose(gla["S"], ret["S"], atol=1e-13)
+    lin = oracle.eager_rollout(LINATTN, S0, q, k, v, None, scale=1.1)
+    ret0 = oracle.eager_rollout(RETNET, S0, q, k, v, np.zeros_like(lam1), scale=1.1)
+    np.testing.assert_allclose(lin["out"], ret0["out"], atol=1e-13)
+    lin0 = oracle.eager_rollout(LINATTN, np.zeros_like(S0), q, k, v, None)
+    prefix = np.cumsum(np.einsum("tnj,tnc->tnjc", k, v), axis=0)
+    np.testing.assert_allclose(lin0["out"], np.einsum("tnjc,tnj->tnc", prefix, q), atol=1e-12)
+    rw = oracle.eager_rollout(RWKV6, S0, q, k, v, np.zeros((T, N, dk)), bonus=np.ones((N, dk)))
+    lin1 = oracle.eager_rollout(LINATTN, S0, q, k, v, None)
+    np.testing.assert_allclose(rw["out"], lin1["out"], atol=1e-12)     # S_{t-1}^T r + (r.k) v = S_t^T r
+
+
+# ---------------------------------------------------------------------------------------------
 # base-plus-log schedule (Algorithm 1, Eq. 4-6): closure under append and merge
 # ---------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+@pytest.mark.parametrize("op", ALL_OPS)
 @pytest.mark.parametrize("cap", [1, 2, 3, 5, 8])
 def test_log_schedule_equals_eager_after_every_append_and_merge(op, cap):
     T, N, dk, dv = 11, 2, 4, 3
@@ -274,7 +328,7 @@ def test_log_schedule_merge_variants():
         logical.decode_step(st, q[0], k[0], v[0], lam[0], beta=beta[0])
 
 
-@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+@pytest.mark.parametrize("op", ALL_OPS)
 @pytest.mark.parametrize("cap", [1, 3, 4])
 def test_paper_cycle_with_fused_merge_step_equals_eager(op, cap):
     """The paper's own cycle: cap appends, then one step that consumes a token AND materialises
