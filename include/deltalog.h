@@ -15,7 +15,12 @@
  *   DELTALOG_GDN    scalar decay per head, delta rule:   b_t = beta_t (v_t - (D(lambda_t) S_{t-1})^T k_t)
  *   DELTALOG_KDA    per-key decay,          delta rule:   same b_t
  *   DELTALOG_RWKV6  per-key decay, b_t = v_t, output read from S_{t-1} plus the bonus term
- * All use a_t = k_t and S_t = D(lambda_t) S_{t-1} + a_t b_t^T (Eq. 3).
+ *   DELTALOG_LINATTN  no decay (the gate pointer is ignored and may be NULL), b_t = v_t; the caller
+ *                     passes the feature-mapped key phi(k_t) as k
+ *   DELTALOG_RETNET   scalar decay per head (lambda = log gamma), b_t = v_t
+ *   DELTALOG_GLA      per-key decay, b_t = v_t
+ * All use a_t = k_t and S_t = D(lambda_t) S_{t-1} + a_t b_t^T (Eq. 3); all but RWKV6 return
+ * scale * S_t^T q_t.  beta is read by GDN / KDA only, u_bonus by RWKV6 only.
  *
  * General rules for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller; descriptor structs are HOST
@@ -30,7 +35,7 @@
  *     on; kernels never trap.  Rows with slot index < 0 are padding and are skipped silently.
  *   - The same slot must not appear twice in one call.
  *   - Supported shapes: d_k == d_v in {64, 128}; 1 <= cap <= 64; klog_dtype == io_dtype;
- *     ulog_dtype == F32 for GDN / KDA and == io_dtype for RWKV6.
+ *     ulog_dtype == F32 for GDN / KDA and == io_dtype for the operators with b_t = v_t.
  */
 #ifndef DELTALOG_H
 #define DELTALOG_H
@@ -41,7 +46,9 @@
 extern "C" {
 #endif
 
-typedef enum { DELTALOG_GDN = 0, DELTALOG_KDA = 1, DELTALOG_RWKV6 = 2 } deltalog_op;
+typedef enum {
+    DELTALOG_GDN = 0, DELTALOG_KDA = 1, DELTALOG_RWKV6 = 2, DELTALOG_LINATTN = 3, DELTALOG_RETNET = 4, DELTALOG_GLA = 5
+} deltalog_op;
 typedef enum { DELTALOG_F32 = 0, DELTALOG_BF16 = 1 } deltalog_dtype;
 
 /* host-side return codes */
@@ -91,8 +98,9 @@ typedef struct {
  * as entry log_len and increments log_len.  Never writes S_base.
  *
  *   q, k, v  [B, H, d]  io_dtype (q is the receptance r for RWKV6)
- *   g        log-decay lambda_t <= 0, fp32: [B, H] for GDN, [B, H, d_k] for KDA / RWKV6
- *   beta     [B, H] fp32 for GDN / KDA; ignored (may be NULL) for RWKV6
+ *   g        log-decay lambda_t <= 0, fp32: [B, H] for GDN / RetNet, [B, H, d_k] for KDA / RWKV6 / GLA;
+ *            ignored (may be NULL) for plain linear attention
+ *   beta     [B, H] fp32 for GDN / KDA; ignored (may be NULL) otherwise
  *   u_bonus  [H, d_k] fp32 for RWKV6; ignored (may be NULL) otherwise
  *   out      [B, H, d_v] io_dtype;  GDN / KDA: scale * S_t^T q_t;
  *            RWKV6: S_{t-1}^T r_t + (r_t . (u_bonus (.) k_t)) v_t

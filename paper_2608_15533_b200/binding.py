@@ -14,7 +14,9 @@ from typing import Optional
 
 import torch
 
-GDN, KDA, RWKV6 = 0, 1, 2
+GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+_DELTA_RULE = (GDN, KDA)            # b = beta (v - S'^T k): U log in fp32
+_VEC_DECAY = (KDA, RWKV6, GLA)      # one log-decay per key channel
 F32, BF16 = 0, 1
 STATUS_LOG_FULL, STATUS_BAD_SLOT, STATUS_TIMEOUT = 1, 2, 4
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_CAP_RANGE, ERR_CUDA, ERR_STATIC_LIMIT = 0, 1, 2, 3, 4, 5
@@ -119,18 +121,18 @@ class Desc:
     cap: int
     io_dtype: int = BF16
     klog_dtype: Optional[int] = None   # default: io_dtype
-    ulog_dtype: Optional[int] = None   # default: F32 for GDN / KDA, io_dtype for RWKV6
+    ulog_dtype: Optional[int] = None   # default: F32 for GDN / KDA, io_dtype where b = v
     scale: float = 1.0
 
     def __post_init__(self):
         if self.klog_dtype is None:
             self.klog_dtype = self.io_dtype
         if self.ulog_dtype is None:
-            self.ulog_dtype = self.io_dtype if self.op == RWKV6 else F32
+            self.ulog_dtype = F32 if self.op in _DELTA_RULE else self.io_dtype
 
     @property
     def d_lambda(self) -> int:
-        return 1 if self.op == GDN else self.d_k
+        return self.d_k if self.op in _VEC_DECAY else 1
 
     def c_struct(self) -> _Desc:
         key = (self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
@@ -250,7 +252,7 @@ class HostStaging:
         self.q = torch.empty(B, desc.H, desc.d_k, dtype=io, device=device)
         self.k = torch.empty_like(self.q)
         self.v = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
-        gshape = (B, desc.H) if desc.op == GDN else (B, desc.H, desc.d_k)
+        gshape = (B, desc.H, desc.d_k) if desc.op in _VEC_DECAY else (B, desc.H)
         self.g = torch.empty(*gshape, dtype=torch.float32, device=device)
         self.beta = torch.empty(B, desc.H, dtype=torch.float32, device=device)
         self.out = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
@@ -259,7 +261,7 @@ class HostStaging:
         return _Staging(*(t.data_ptr() for t in (self.q, self.k, self.v, self.g, self.beta, self.out)))
 
     def h2d_bytes(self, desc: Desc) -> int:
-        ts = [self.q, self.k, self.v, self.g] + ([] if desc.op == RWKV6 else [self.beta])
+        ts = [self.q, self.k, self.v, self.g] + ([self.beta] if desc.op in _DELTA_RULE else [])
         return sum(t.numel() * t.element_size() for t in ts)
 
     def d2h_bytes(self) -> int:

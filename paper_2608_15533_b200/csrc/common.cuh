@@ -13,6 +13,16 @@ constexpr int kThreads = 256;  // every kernel in this library runs 256-thread C
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCap = 64;
 
+// What the kernels need to know about an operator of Table 1.  The additive family shares kernels:
+// plain linear attention runs the RetNet instantiation with a null gate pointer (lambda == 0).
+template <int OP>
+struct OpTraits {
+    static constexpr bool kVecDecay = (OP == DELTALOG_KDA || OP == DELTALOG_RWKV6 || OP == DELTALOG_GLA);
+    static constexpr bool kDeltaRule = (OP == DELTALOG_GDN || OP == DELTALOG_KDA);  // b = beta (v - S'^T k), else b = v
+    static constexpr bool kPostReadout = (OP != DELTALOG_RWKV6);  // output read from S_t (scaled); RWKV6 reads S_{t-1}
+    static constexpr bool kBonus = (OP == DELTALOG_RWKV6);
+};
+
 template <int DT> struct DType;
 template <> struct DType<DELTALOG_F32> { using type = float; };
 template <> struct DType<DELTALOG_BF16> { using type = __nv_bfloat16; };

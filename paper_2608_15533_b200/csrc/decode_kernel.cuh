@@ -27,7 +27,7 @@ __host__ __device__ constexpr int decode_threads() {
 
 template <int D, typename IO, typename UL>
 __host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
-    const size_t dl = (op == DELTALOG_GDN) ? 1 : D;
+    const size_t dl = (op == DELTALOG_GDN || op == DELTALOG_RETNET || op == DELTALOG_LINATTN) ? 1 : D;
     size_t bytes = 0;
     bytes += sizeof(float) * D * 5;                 // q, k (raw), mul_k, mul_q, lbar'/u scratch
     bytes += sizeof(float) * D;                     // lbar_old (vector ops)
@@ -47,8 +47,9 @@ template <int OP, int D, typename IO, typename UL>
 __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPLE_CTAS : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
     constexpr int NT = decode_threads<D>();
     constexpr int NW = NT / 32;
-    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
-    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
+    constexpr bool kPost = OpTraits<OP>::kPostReadout;
+    constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4;          // float4 columns per state row
     constexpr int RL = NT / C4;        // rows covered by one pass of the CTA
@@ -112,11 +113,11 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
         k_raw = kg[tid];
         const float kv = to_f32(k_raw);
         const float lold = (len > 0) ? Lg[(size_t)(len - 1) * DL + (kVecDecay ? tid : 0)] : 0.f;
-        lnew = lold + gg[kVecDecay ? tid : 0];
+        lnew = lold + (tk.g ? gg[kVecDecay ? tid : 0] : 0.f);  // no gate: plain linear attention
         q_s[tid] = qv;
         k_s[tid] = kv;
-        lold_s[tid] = kDelta ? lnew : lold;  // the decay level the replay coefficients refer to
-        const float e = expf(kDelta ? lnew : lold);
+        lold_s[tid] = kPost ? lnew : lold;  // the decay level the replay coefficients refer to
+        const float e = expf(kPost ? lnew : lold);
         mk_s[tid] = e * kv;
         mq_s[tid] = e * qv;
     }
@@ -147,7 +148,7 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kDelta ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -190,7 +191,7 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
         if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
     } else if (active) {
         const IO v_raw = vg[c];
-        og[c] = from_f32<IO>(fmaf(scal_s[0], to_f32(v_raw), y));
+        og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], to_f32(v_raw), y));
         Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
     }
     if (tid < D) {

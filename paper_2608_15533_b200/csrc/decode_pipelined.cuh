@@ -43,7 +43,7 @@ __host__ __device__ constexpr int align_up(int x, int a) { return (x + a - 1) / 
 // Byte offsets inside one aux-ring stage (all multiples of 16).
 template <int OP, int D, typename IO, typename UL>
 struct AuxLayout {
-    static constexpr bool kVec = (OP != DELTALOG_GDN);
+    static constexpr bool kVec = OpTraits<OP>::kVecDecay;
     static constexpr int DL = kVec ? D : 1;
     int K, U, L, q, k, v, g, bonus, meta, bytes;
     __host__ __device__ explicit AuxLayout(int cap) {
@@ -171,8 +171,9 @@ struct RingPos {  // position in a ring of n stages: stage index and phase parit
 template <int OP, int D, typename IO, typename UL>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
-    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
-    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
+    constexpr bool kPost = OpTraits<OP>::kPostReadout;
+    constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4;
     constexpr int RL = kPipeConsumers / C4;          // row groups of the stream group
@@ -292,7 +293,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         if (st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
                         flags = kMetaFull;
                     }
-                    if (!kVecDecay) gs = tk.g[item];
+                    if (!kVecDecay && tk.g) gs = tk.g[item];  // no gate: plain linear attention
                     if (kDelta) bt = tk.beta[item];
                 }
             }
@@ -443,9 +444,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         const float lnew = lold + (kVecDecay ? g_a[gtid] : __int_as_float(meta.z));
                         q_s[gtid] = qv;
                         k_s[gtid] = kv;
-                        lbar_s[gtid] = kDelta ? lnew : lold;  // the decay level the readouts refer to
+                        lbar_s[gtid] = kPost ? lnew : lold;  // the decay level the readouts refer to
                         sl[oLN + gtid] = lnew;                // the level stored with the appended entry
-                        const float e = expf(kDelta ? lnew : lold);
+                        const float e = expf(kPost ? lnew : lold);
                         sl[oMK + gtid] = e * kv;
                         sl[oMQ + gtid] = e * qv;
                     }
@@ -505,9 +506,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     if (gwarp == kHalf - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
                         float d = 0.f;
                         float bw[EPL];
-                        if (!kDelta) load_vec<float, EPL>(bonus_a + lane * EPL, bw);
+                        if (!kPost) load_vec<float, EPL>(bonus_a + lane * EPL, bw);
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) d = fmaf(kDelta ? qv[e] : qv[e] * bw[e], kv[e], d);
+                        for (int e = 0; e < EPL; ++e) d = fmaf(kPost ? qv[e] : qv[e] * bw[e], kv[e], d);
                         d = warp_sum(d);
                         if (lane == 0) sl[oSC] = d;
                     }
@@ -566,7 +567,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         og[c] = from_f32<IO>(st.scale * fmaf(sl[oSC], bval, yq));
                     } else {
                         Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
-                        og[c] = from_f32<IO>(fmaf(sl[oSC], to_f32(v_raw), yq));
+                        og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(sl[oSC], to_f32(v_raw), yq));
                     }
                     (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[c] = k_a[c];
                     if (kVecDecay) st.decay_log[(unit * cap + len) * DL + c] = sl[oLN + c];

@@ -1,6 +1,9 @@
 // C ABI of the DeltaLog decode library: host-side argument validation and kernel dispatch.
 // Declarations and the contract of every entry point are in include/deltalog.h.
 #include <atomic>
+#include <map>
+#include <mutex>
+#include <utility>
 #include <cstdint>
 #include <type_traits>
 
@@ -19,16 +22,21 @@ std::atomic<uint64_t> g_launches{0};
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Operator facts needed on the host side (Table 1).
+bool op_delta_rule(int op) { return op == DELTALOG_GDN || op == DELTALOG_KDA; }
+bool op_has_gate(int op) { return op != DELTALOG_LINATTN; }
+bool op_vec_decay(int op) { return op == DELTALOG_KDA || op == DELTALOG_RWKV6 || op == DELTALOG_GLA; }
+
 int validate_desc(const deltalog_desc *d) {
     if (!d) return DELTALOG_ERR_INVALID_ARG;
-    if (d->op < DELTALOG_GDN || d->op > DELTALOG_RWKV6) return DELTALOG_ERR_INVALID_ARG;
+    if (d->op < DELTALOG_GDN || d->op > DELTALOG_GLA) return DELTALOG_ERR_INVALID_ARG;
     if (d->num_slots <= 0 || d->H <= 0) return DELTALOG_ERR_INVALID_ARG;
     if (d->io_dtype != DELTALOG_F32 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->klog_dtype != DELTALOG_F32 && d->klog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->ulog_dtype != DELTALOG_F32 && d->ulog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->d_k != d->d_v || (d->d_k != 64 && d->d_k != 128)) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     if (d->klog_dtype != d->io_dtype) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    const int want_u = (d->op == DELTALOG_RWKV6) ? d->io_dtype : (int)DELTALOG_F32;
+    const int want_u = op_delta_rule(d->op) ? (int)DELTALOG_F32 : d->io_dtype;  // b = v is lossless in the I/O dtype
     if (d->ulog_dtype != want_u) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     if (d->cap < 1 || d->cap > kMaxCap) return DELTALOG_ERR_CAP_RANGE;
     return DELTALOG_OK;
@@ -45,9 +53,11 @@ int validate_state(const deltalog_state *s) {
 int validate_token(const deltalog_desc *d, const void *q, const void *k, const void *v, const float *g,
                    const float *beta, const float *u_bonus, int32_t B, const void *out) {
     if (B < 0) return DELTALOG_ERR_INVALID_ARG;
-    if (!q || !k || !v || !g || !out) return DELTALOG_ERR_INVALID_ARG;
-    if (d->op == DELTALOG_RWKV6 ? !u_bonus : !beta) return DELTALOG_ERR_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(g))
+    if (!q || !k || !v || !out) return DELTALOG_ERR_INVALID_ARG;
+    if (op_has_gate(d->op) && !g) return DELTALOG_ERR_INVALID_ARG;
+    if (op_delta_rule(d->op) && !beta) return DELTALOG_ERR_INVALID_ARG;
+    if (d->op == DELTALOG_RWKV6 && !u_bonus) return DELTALOG_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (op_has_gate(d->op) && !aligned16(g)))
         return DELTALOG_ERR_INVALID_ARG;
     return DELTALOG_OK;
 }
@@ -72,12 +82,25 @@ int finish_launch() {
     return cudaGetLastError() == cudaSuccess ? DELTALOG_OK : DELTALOG_ERR_CUDA;
 }
 
-// Raise the dynamic shared-memory limit of a kernel once per process when it needs more than 48 KiB.
+// Raise the dynamic shared-memory limit of a kernel when a launch needs more than 48 KiB.  The limit
+// only ever grows (per device), and it is raised to what launches have asked for, not to the device
+// maximum: a kernel with static shared memory cannot be granted the whole opt-in size as dynamic.
 template <typename K>
 int ensure_smem(K kernel, size_t bytes) {
     if (bytes <= 48 * 1024) return DELTALOG_OK;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    static std::mutex mu;
+    static std::map<std::pair<int, const void *>, size_t> granted;  // (device, kernel) -> bytes granted
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const auto key = std::make_pair(dev, reinterpret_cast<const void *>(kernel));
+    std::lock_guard<std::mutex> lock(mu);
+    size_t &g = granted[key];
+    if (bytes <= g) return DELTALOG_OK;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+        cudaGetLastError();  // not sticky: leave the runtime clean for the caller
         return DELTALOG_ERR_CUDA;
+    }
+    g = bytes;
     return DELTALOG_OK;
 }
 
@@ -109,7 +132,7 @@ int env_int(const char *name, int dflt) {
 
 template <int OP, int D, typename IO>
 int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
     static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
     static const int env_base = env_int("DELTALOG_BASE_STAGES", 0);
@@ -121,7 +144,7 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
     // every unit's snapshot row to start on a 16-byte boundary: cap % 4 == 0 for GDN.
     // Head size 64: a unit is a single 16 KiB chunk and the per-unit hand-overs of the pipeline cost
     // more than they hide, so the one-CTA-per-unit kernel is the faster one there (measured).
-    bool pipelined = impl != 1 && dev.sms > 0 && (OP != DELTALOG_GDN || st.cap % 4 == 0) && (D == 128 || impl == 2);
+    bool pipelined = impl != 1 && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0) && (D == 128 || impl == 2);
     PipeCfg cfg{0, 0};
     int ctas = env_ctas > 0 ? env_ctas : 1;
     if (pipelined) {
@@ -159,7 +182,7 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
 template <int OP, int D, typename IO>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
-    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     const size_t smem = merge_smem_bytes<D>(st.cap);
     // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
     // call over a whole batch whose fills are staggered) most units are skipped: eight per CTA.
@@ -178,7 +201,7 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
 
 template <int OP, int D, typename IO>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    using UL = typename std::conditional<OP == DELTALOG_RWKV6, IO, float>::type;
+    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     auto kernel = decode_merge_step_kernel<OP, D, IO, UL>;
     const size_t smem = fused_step_smem_bytes<D>(st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
@@ -200,6 +223,10 @@ int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenA
             DELTALOG_DISPATCH_D(DELTALOG_GDN, d_, io_, CALL);                                \
         } else if (op_ == DELTALOG_KDA) {                                                    \
             DELTALOG_DISPATCH_D(DELTALOG_KDA, d_, io_, CALL);                                \
+        } else if (op_ == DELTALOG_RETNET || op_ == DELTALOG_LINATTN) {                      \
+            DELTALOG_DISPATCH_D(DELTALOG_RETNET, d_, io_, CALL); /* linear attention: null gate */ \
+        } else if (op_ == DELTALOG_GLA) {                                                    \
+            DELTALOG_DISPATCH_D(DELTALOG_GLA, d_, io_, CALL);                                \
         } else {                                                                             \
             DELTALOG_DISPATCH_D(DELTALOG_RWKV6, d_, io_, CALL);                              \
         }                                                                                    \
@@ -227,7 +254,7 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
-    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_DECODE(OP, D, IO) return launch_decode<OP, D, IO>(st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
@@ -244,7 +271,7 @@ int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
-    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_FUSED(OP, D, IO) return launch_fused_step<OP, D, IO>(st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_FUSED);
@@ -273,7 +300,7 @@ int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, cons
     if (!S || !aligned16(S)) return DELTALOG_ERR_INVALID_ARG;
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
-    const TokenArgs tk{q, k, v, g, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_EAGER(OP, D, IO) return launch_eager<OP, D, IO>(S, desc, status, tk, s)
     DELTALOG_DISPATCH(desc, CALL_EAGER);
@@ -287,21 +314,23 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
                               const float *host_beta, const float *u_bonus,
                               const int32_t *slot_idx, int32_t B, void *host_out, void *stream) {
     if (int rc = validate_desc(desc)) return rc;
-    if (!staging || !host_q || !host_k || !host_v || !host_g || !host_out) return DELTALOG_ERR_INVALID_ARG;
-    if (desc->op != DELTALOG_RWKV6 && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
+    if (!staging || !host_q || !host_k || !host_v || !host_out) return DELTALOG_ERR_INVALID_ARG;
+    if (op_has_gate(desc->op) && (!host_g || !staging->g)) return DELTALOG_ERR_INVALID_ARG;
+    if (op_delta_rule(desc->op) && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
     if (B < 0) return DELTALOG_ERR_INVALID_ARG;
     if (B == 0) return DELTALOG_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t units = (size_t)B * desc->H;
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
     const size_t vec = units * desc->d_k * esz;
-    const size_t gbytes = units * (desc->op == DELTALOG_GDN ? 1 : desc->d_k) * sizeof(float);
-    if (!staging->q || !staging->k || !staging->v || !staging->g || !staging->out) return DELTALOG_ERR_INVALID_ARG;
+    const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
+    if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
     bool ok = cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (desc->op != DELTALOG_RWKV6)
+    if (op_has_gate(desc->op))
+        ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    if (op_delta_rule(desc->op))
         ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s) ==
                        cudaSuccess;
     if (!ok) return DELTALOG_ERR_CUDA;
@@ -319,10 +348,11 @@ int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltal
                                          const float *host_g, const float *host_beta, const float *u_bonus,
                                          const int32_t *slot_idx, int32_t B, void *host_out) {
     if (int rc = validate_desc(desc)) return rc;
-    if (!staging || !lane || !host_q || !host_k || !host_v || !host_g || !host_out) return DELTALOG_ERR_INVALID_ARG;
+    if (!staging || !lane || !host_q || !host_k || !host_v || !host_out) return DELTALOG_ERR_INVALID_ARG;
     if (!lane->in_done || !lane->compute_done || !lane->out_done) return DELTALOG_ERR_INVALID_ARG;
-    if (desc->op != DELTALOG_RWKV6 && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
-    if (!staging->q || !staging->k || !staging->v || !staging->g || !staging->out) return DELTALOG_ERR_INVALID_ARG;
+    if (op_has_gate(desc->op) && (!host_g || !staging->g)) return DELTALOG_ERR_INVALID_ARG;
+    if (op_delta_rule(desc->op) && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
+    if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
     if (B < 0) return DELTALOG_ERR_INVALID_ARG;
     if (B == 0) return DELTALOG_OK;
     cudaStream_t s_in = static_cast<cudaStream_t>(lane->copy_in_stream);
@@ -334,14 +364,15 @@ int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltal
     const size_t units = (size_t)B * desc->H;
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
     const size_t vec = units * desc->d_k * esz;
-    const size_t gbytes = units * (desc->op == DELTALOG_GDN ? 1 : desc->d_k) * sizeof(float);
+    const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
     // copy-in stream: the staging inputs are free once the kernel that last read them is done
     bool ok = cudaStreamWaitEvent(s_in, e_cmp, 0) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    if (desc->op != DELTALOG_RWKV6)
+    if (op_has_gate(desc->op))
+        ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    if (op_delta_rule(desc->op))
         ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s_in) ==
                        cudaSuccess;
     ok = ok && cudaEventRecord(e_in, s_in) == cudaSuccess;

@@ -14,8 +14,9 @@ namespace deltalog {
 template <int OP, int D, typename IO>
 __global__ void __launch_bounds__(kThreads, 2)
 eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *status, TokenArgs tk) {
-    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
-    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
+    constexpr bool kPost = OpTraits<OP>::kPostReadout;
+    constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL, EPL = D / 32;
 
@@ -39,7 +40,7 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
     if (tid < D) {
         q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[row * D + tid]);
         k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[row * D + tid]);
-        a_s[tid] = expf(tk.g[row * DL + (kVecDecay ? tid : 0)]);
+        a_s[tid] = tk.g ? expf(tk.g[row * DL + (kVecDecay ? tid : 0)]) : 1.f;  // no gate: plain linear attention
     }
     __syncthreads();
     if (warp == 0) {
@@ -47,7 +48,7 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kDelta ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -58,10 +59,10 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
 #pragma unroll
     for (int p = 0; p < NP; ++p) {
         const int r = p * RL + rl;
-        if (kDelta) {  // decay first; both readouts are taken on the decayed state
+        if (kPost) {  // decay first; the readouts are taken on the decayed state
             const float a = a_s[r];
             s[p] = make_float4(a * s[p].x, a * s[p].y, a * s[p].z, a * s[p].w);
-            ak = fma4(k_s[r], s[p], ak);
+            if (kDelta) ak = fma4(k_s[r], s[p], ak);
         }
         aq = fma4(q_s[r], s[p], aq);  // RWKV6: readout on the old state
     }
@@ -87,7 +88,7 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
         if (active) {
             const float vv = to_f32(vg[c]);
             b_s[c] = vv;
-            og[c] = from_f32<IO>(fmaf(qk_s, vv, y));
+            og[c] = from_f32<IO>((kPost ? scale : 1.f) * fmaf(qk_s, vv, y));
         }
         __syncthreads();
     }
@@ -97,7 +98,7 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
     for (int p = 0; p < NP; ++p) {
         const int r = p * RL + rl;
         float4 x = s[p];
-        if (!kDelta) {
+        if (!kPost) {
             const float a = a_s[r];
             x = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
         }

@@ -25,8 +25,9 @@ __host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
 
 template <int OP, int D, typename IO, typename UL>
 __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
-    constexpr bool kDelta = (OP != DELTALOG_RWKV6);
-    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
+    constexpr bool kPost = OpTraits<OP>::kPostReadout;
+    constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL, EPL = D / 32;
 
@@ -65,7 +66,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     // lref: the decay level the state is materialised at -- lbar' for the delta rule (both readouts
     // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
     if (!kVecDecay) {
-        const float lref = (len > 0 ? lold[0] : 0.f) + gg[0];
+        const float lref = (len > 0 ? lold[0] : 0.f) + (tk.g ? gg[0] : 0.f);  // no gate: plain linear attention
         for (int x = tid * 4; x < len * D; x += kThreads * 4) {
             const float wi = expf(lref - Lg[x / D]);
             float kv[4], uv[4];
@@ -77,7 +78,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     } else {
         for (int x = tid; x < len * D; x += kThreads) {
             const int i = x / D, j = x % D;
-            const float lref = lold[j] + (kDelta ? gg[j] : 0.f);
+            const float lref = lold[j] + (kPost ? gg[j] : 0.f);
             A_s[x] = expf(lref - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);
             U_s[x] = to_f32(Ug[x]);
         }
@@ -85,10 +86,10 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     const IO *vg = static_cast<const IO *>(tk.v) + row * D;
     if (tid < D) {
         const int jl = kVecDecay ? tid : 0;
-        const float lo = len > 0 ? lold[jl] : 0.f, lam = gg[jl];
+        const float lo = len > 0 ? lold[jl] : 0.f, lam = tk.g ? gg[jl] : 0.f;
         q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[row * D + tid]);
         k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[row * D + tid]);
-        e_s[tid] = expf(kDelta ? lo + lam : lo);
+        e_s[tid] = expf(kPost ? lo + lam : lo);
         w_s[tid] = expf(lam);
     }
     __syncthreads();
@@ -98,7 +99,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kDelta ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -147,7 +148,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
         if (active) {
             const float vv = to_f32(vg[c]);
             b_s[c] = vv;
-            og[c] = from_f32<IO>(fmaf(scal_s[0], vv, y));
+            og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], vv, y));
         }
         __syncthreads();
     }
@@ -158,7 +159,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     for (int p = 0; p < NP; ++p) {
         const int r = rl * NP + p;
         float4 x = s[p];
-        if (!kDelta) {
+        if (!kPost) {
             const float a = w_s[r];
             x = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
         }

@@ -25,7 +25,7 @@ constexpr size_t merge_smem_bytes(int cap) {
 template <int OP, int D, typename IO, typename UL, int PACK>
 __global__ void __launch_bounds__(kThreads, DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
-    constexpr bool kVecDecay = (OP != DELTALOG_GDN);
+    constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL;
 

@@ -51,7 +51,7 @@ extern "C" int deltalog_decode_step_host_static(const deltalog_desc *desc, const
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
     const size_t qk = round256(units * (size_t)desc->d_k * esz);
     const size_t vo = round256(units * (size_t)desc->d_v * esz);
-    const size_t gb = round256(units * (size_t)(desc->op == DELTALOG_GDN ? 1 : desc->d_k) * sizeof(float));
+    const size_t gb = round256(units * (size_t)(desc->op == DELTALOG_KDA || desc->op == DELTALOG_RWKV6 || desc->op == DELTALOG_GLA ? desc->d_k : 1) * sizeof(float));
     const size_t bb = round256(units * sizeof(float));
     if (2 * qk + 2 * vo + gb + bb > (size_t)DELTALOG_STATIC_STAGING_BYTES) return DELTALOG_ERR_STATIC_LIMIT;
 

@@ -61,7 +61,10 @@ class Recorded:
         self.q.append(f64(tok["q"][b, h]))
         self.k.append(f64(tok["k"][b, h]))
         self.v.append(f64(tok["v"][b, h]))
-        self.g.append(f64(tok["g"][b, h]).reshape(len(self.units), -1))
+        if tok["g"] is not None:
+            self.g.append(f64(tok["g"][b, h]).reshape(len(self.units), -1))
+        else:  # plain linear attention has no gate
+            self.g.append(np.zeros((len(self.units), 1)))
         if tok["beta"] is not None:
             self.beta.append(f64(tok["beta"][b, h]))
         self.out.append(f64(out[b, h]))

@@ -370,3 +370,13 @@ def test_overlapped_host_entry_point_matches_device_entry_point_over_a_cycle():
     torch.cuda.synchronize()
     assert torch.equal(s_dev.S_base, s_host.S_base) and torch.equal(s_dev.U_log, s_host.U_log)
     assert torch.equal(s_dev.log_len, s_host.log_len)
+
+
+@pytest.mark.parametrize("op", [GDN, KDA])
+def test_predicate_merge_at_capacity_64_head_size_128(op):
+    """The packed predicate merge needs more than 48 KiB of dynamic shared memory here, beside its
+    static arrays."""
+    wl = small(op, 128, torch.bfloat16, batch=5, H=3, steps=140)
+    rec, state, S0u, bonus = run_deltalog(wl, 64, DEV, units=[(0, 0), (2, 1), (4, 2)])
+    assert 64 in rec.state_at and 128 in rec.state_at
+    check_rollout(wl, rec, oracle_for(wl, rec, S0u, bonus))

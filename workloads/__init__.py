@@ -24,8 +24,8 @@ from typing import Dict, Iterator, Optional, Tuple
 
 import torch
 
-GDN, KDA, RWKV6 = 0, 1, 2
-OP_NAMES = {GDN: "gdn", KDA: "kda", RWKV6: "rwkv6"}
+GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+OP_NAMES = {GDN: "gdn", KDA: "kda", RWKV6: "rwkv6", LINATTN: "linattn", RETNET: "retnet", GLA: "gla"}
 
 
 @dataclass(frozen=True)
@@ -51,7 +51,7 @@ class Workload:
 
     @property
     def d_lambda(self) -> int:
-        return 1 if self.op == GDN else self.d
+        return self.d if self.op in (KDA, RWKV6, GLA) else 1
 
     @property
     def units(self) -> int:
@@ -116,13 +116,31 @@ class TokenSource:
             g = -torch.exp(self._randn(B, H, d).mul_(0.5).sub_(0.5))
             _ = self._randn(B, H)  # keeps the draw order uniform across operators
             beta = None
+        elif wl.op in (LINATTN, RETNET, GLA):
+            # additive family: L2-normalised q, k (for plain linear attention after the positive feature
+            # map elu(x) + 1, which the caller of the library applies); RetNet's decay is the fixed
+            # per-head gamma_h = 1 - 2^(-5-h mod 8); GLA's gate is drawn like KDA's; no beta
+            if wl.op == LINATTN:
+                q, k = torch.nn.functional.elu(q) + 1.0, torch.nn.functional.elu(k) + 1.0
+            q, k = _l2_normalise(q), _l2_normalise(k)
+            noise = self._randn(B, H, d)   # drawn for every operator of the family: uniform draw order
+            if wl.op == GLA:
+                g = -torch.nn.functional.softplus(noise)
+            elif wl.op == RETNET:
+                h = torch.arange(H, device=self.device, dtype=torch.float32) % 8
+                g = torch.log1p(-torch.pow(2.0, -5.0 - h)).expand(B, H)
+            else:
+                g = None
+            _ = self._randn(B, H)
+            beta = None
         else:
             q, k = _l2_normalise(q), _l2_normalise(k)
             gate_shape = (B, H) if wl.op == GDN else (B, H, d)
             g = -torch.nn.functional.softplus(self._randn(*gate_shape))
             beta = torch.sigmoid(self._randn(B, H))
         dt = wl.io_dtype
-        return {"q": q.to(dt), "k": k.to(dt), "v": v.to(dt), "g": g.contiguous(), "beta": beta}
+        return {"q": q.to(dt), "k": k.to(dt), "v": v.to(dt), "g": g.contiguous() if g is not None else None,
+                "beta": beta}
 
     def tokens(self, n: int) -> Iterator[Dict[str, Optional[torch.Tensor]]]:
         for _ in range(n):
