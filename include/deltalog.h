@@ -138,6 +138,17 @@ int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const
                    int32_t n, int32_t only_if_full, void *stream);
 
 /*
+ * Slot lifecycle (Section 4, state-slot lifecycle): hand the n listed slots (slots 0..n-1 if slot_idx
+ * is NULL) to new requests.  The log of every head of a listed slot is emptied (log_len <- 0, which
+ * also clears lbar); pending entries are discarded, not folded.  With S_init != NULL (device,
+ * [n, H, d_k, d_v] fp32, e.g. the state a prefill produced) the base of listed slot i becomes
+ * S_init[i]; with S_init == NULL the base is left as it is.  Other slots are untouched.  Slot
+ * indices < 0 are skipped, indices >= num_slots set DELTALOG_STATUS_BAD_SLOT and are skipped.
+ */
+int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state, const int32_t *slot_idx,
+                         int32_t n, const float *S_init, void *stream);
+
+/*
  * The eager dense comparator (Section 2.3): the same token update applied directly to a dense
  * state S [num_slots, H, d_k, d_v] fp32, which is read and rewritten in full on every call.
  * Token arguments and `out` as for deltalog_decode_step; `status` (may be NULL) receives

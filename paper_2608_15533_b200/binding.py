@@ -28,7 +28,7 @@ _DT_TO_TORCH = {F32: torch.float32, BF16: torch.bfloat16}
 LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
 
 EXPORTS = (
-    "deltalog_decode_step", "deltalog_decode_merge_step", "deltalog_merge", "deltalog_eager_step", "deltalog_decode_step_host",
+    "deltalog_decode_step", "deltalog_decode_merge_step", "deltalog_merge", "deltalog_reset_slots", "deltalog_eager_step", "deltalog_decode_step_host",
     "deltalog_decode_step_host_static", "deltalog_decode_step_host_overlapped",
     "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
 )
@@ -78,6 +78,8 @@ def load_library() -> ctypes.CDLL:
         lib.deltalog_decode_merge_step.argtypes = lib.deltalog_decode_step.argtypes
         lib.deltalog_merge.restype = ctypes.c_int
         lib.deltalog_merge.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State), vp, i32, i32, vp]
+        lib.deltalog_reset_slots.restype = ctypes.c_int
+        lib.deltalog_reset_slots.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State), vp, i32, vp, vp]
         lib.deltalog_eager_step.restype = ctypes.c_int
         lib.deltalog_eager_step.argtypes = [ctypes.POINTER(_Desc)] + [vp] * 8 + [i32, vp, vp, vp]
         lib.deltalog_decode_step_host.restype = ctypes.c_int
@@ -228,6 +230,17 @@ def merge(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None, only
     rc = load_library().deltalog_merge(ctypes.byref(d), ctypes.byref(s), _ptr(slot_idx), int(n),
                                        int(bool(only_if_full)), _stream(stream))
     _check(rc, "deltalog_merge")
+
+
+def reset_slots(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None, S_init=None, stream=None) -> None:
+    """``deltalog_reset_slots``: empty the logs of the listed slots (all when ``slot_idx`` is None) and,
+    with ``S_init [n,H,d_k,d_v]``, install new base states (prefill hand-off)."""
+    if n is None:
+        n = desc.num_slots if slot_idx is None else slot_idx.numel()
+    d, s = desc.c_struct(), state.c_struct()
+    rc = load_library().deltalog_reset_slots(ctypes.byref(d), ctypes.byref(s), _ptr(slot_idx), int(n),
+                                             _ptr(S_init), _stream(stream))
+    _check(rc, "deltalog_reset_slots")
 
 
 def eager_step(desc: Desc, S: torch.Tensor, q, k, v, g, beta=None, u_bonus=None, slot_idx=None, out=None,

@@ -293,6 +293,21 @@ int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const
     return DELTALOG_ERR_INVALID_ARG;
 }
 
+int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state, const int32_t *slot_idx,
+                         int32_t n, const float *S_init, void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
+    if (n < 0 || (!slot_idx && n > desc->num_slots) || (S_init && !aligned16(S_init))) return DELTALOG_ERR_INVALID_ARG;
+    if (n == 0) return DELTALOG_OK;
+    const StateArgs st = make_state_args(desc, state);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (desc->d_k == 64)
+        reset_slots_kernel<64><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+    else
+        reset_slots_kernel<128><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+    return finish_launch();
+}
+
 int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, const void *k,
                         const void *v, const float *g, const float *beta, const float *u_bonus,
                         const int32_t *slot_idx, int32_t B, void *out, int32_t *status, void *stream) {

@@ -120,4 +120,19 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     }
 }
 
+// Slot hand-over: empty the log of every head of the listed slots and, if given, install a new base.
+template <int D>
+__global__ void __launch_bounds__(kThreads) reset_slots_kernel(StateArgs st, const int32_t *slot_idx, const float *S_init) {
+    const int i = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    int slot;
+    if (!resolve_slot(slot_idx, i, st.num_slots, st.status, threadIdx.x, slot)) return;
+    const size_t unit = (size_t)slot * st.H + h;
+    if (S_init) {
+        const float4 *src = reinterpret_cast<const float4 *>(S_init + ((size_t)i * st.H + h) * D * D);
+        float4 *dst = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
+        for (int x = threadIdx.x; x < D * D / 4; x += kThreads) dst[x] = src[x];
+    }
+    if (threadIdx.x == 0) st.log_len[unit] = 0;
+}
+
 }  // namespace deltalog
