@@ -14,6 +14,7 @@
 #include "eager_kernel.cuh"
 #include "fused_step_kernel.cuh"
 #include "merge_kernel.cuh"
+#include "merge_tc_kernel.cuh"
 
 namespace deltalog {
 namespace {
@@ -183,6 +184,22 @@ template <int OP, int D, typename IO>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
     using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
+    // DELTALOG_MERGE_TC = 1 (head size 128, no predicate): the contraction over the log entries runs
+    // on the tensor cores (tcgen05, tf32 x 3).  Off by default: it executes a fraction of the
+    // instructions, but with one unit per CTA the extra hand-overs (raw entries -> operands -> MMA ->
+    // tensor-memory load) lengthen each CTA's dependent chain by more than the fp32 pipe costs
+    // (measured on configuration 1: 110 / 119 / 142 / 215 us at capacity 4 / 16 / 32 / 64 against
+    // 85 / 99 / 130 / 195 us for the packed-FMA kernel).
+    static const int use_tc = env_int("DELTALOG_MERGE_TC", 0);
+    if constexpr (D == kTcD) {
+        if (use_tc && !only_if_full) {
+            auto kernel = merge_tc_kernel<OP, IO, UL>;
+            const size_t bytes = merge_tc_smem_bytes<OP, IO, UL>(st.cap);
+            if (int rc = ensure_smem(kernel, bytes)) return rc;
+            kernel<<<n * st.H, kThreads, bytes, stream>>>(st, slot_idx, only_if_full);
+            return finish_launch();
+        }
+    }
     const size_t smem = merge_smem_bytes<D>(st.cap);
     // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
     // call over a whole batch whose fills are staggered) most units are skipped: eight per CTA.
