@@ -271,8 +271,9 @@ def time_paper_cycle(rig: Rig, steps: int):
     """The paper's own cycle (Algorithm 1): cap appends, then one fused step that consumes a token and
     materialises; cap + 1 tokens per dense write.  Uniform batch: one launch per step.  Staggered batch
     (fills uniform on 0..cap): every step is two launches over phase-split batches -- the append
-    call sees slot -1 for the rows whose log is full, the fused-step call for all the others; the
-    host knows each row's phase from its step counter, so the lists are precomputed for one period.
+    call sees slot -1 for the rows whose log is full, the fused-step call gets exactly those rows as
+    its batch; the host knows each row's phase from its step counter, so the lists are precomputed for
+    one period.
     Timed as CUDA-graph replays of whole cycles; on a single-layer uniform batch the fused step alone
     is then timed over plain launches with one event pair per cycle.
     Returns (steps timed, total ms, mean ms of a fused-step launch or None)."""
@@ -284,17 +285,25 @@ def time_paper_cycle(rig: Rig, steps: int):
     for layer in range(rig.layers):
         rig.merge(layer, only_if_full=False)
     dl = rig.dl
-    app_lists = mrg_lists = None
+    app_lists = blocks = slots_sorted = None
     if rig.staggered:
-        delay = workloads.fill_offsets(rig.wl, M).to(rig.device)   # row b starts `delay` steps late: fill cap - delay
-        skip = torch.full_like(rig.slot_idx, -1)
+        # Rows are relabelled so that the rows of one phase are consecutive (the token tensors are
+        # synthetic, the relabelling only permutes which slot a row addresses): the merge-phase batch
+        # of a step is then a contiguous slice of the token tensors, as a runtime with separate append
+        # and merge queues would hand it over.
+        delay, order = torch.sort(workloads.fill_offsets(rig.wl, M).to(rig.device))  # row b starts `delay` steps late
+        slots_sorted = rig.slot_idx[order].contiguous()
+        skip = torch.full_like(slots_sorted, -1)
         for t in range(cap):
-            slots = torch.where(delay <= t, rig.slot_idx, skip)
+            slots = torch.where(delay <= t, slots_sorted, skip)
             for layer in range(rig.layers):
                 rig.decode(t, layer, slot_idx=slots)
-        full_at = [((tau - delay) % M) == 0 for tau in range(M)]     # row is full before step tau of a period
-        app_lists = [torch.where(f, skip, rig.slot_idx) for f in full_at]
-        mrg_lists = [torch.where(f, rig.slot_idx, skip) for f in full_at]
+        app_lists, blocks = [], []
+        for tau in range(M):                                   # a row is full before step tau iff delay == tau
+            full = delay == tau
+            app_lists.append(torch.where(full, skip, slots_sorted))
+            idx = torch.nonzero(full).flatten()
+            blocks.append((int(idx[0]), int(idx[-1]) + 1) if idx.numel() else None)
 
     def one(t, layer):
         tok = rig.rings[layer][t % rig.RING]
@@ -302,7 +311,11 @@ def time_paper_cycle(rig: Rig, steps: int):
         kw = dict(beta=tok["beta"], u_bonus=rig.bonus[layer], out=rig.out)
         if rig.staggered:
             dl.decode_step(*args, slot_idx=app_lists[t % M], **kw)
-            dl.decode_merge_step(*args, slot_idx=mrg_lists[t % M], **kw)
+            if blocks[t % M] is not None:
+                lo, hi = blocks[t % M]
+                dl.decode_merge_step(rig.desc, rig.states[layer], tok["q"][lo:hi], tok["k"][lo:hi], tok["v"][lo:hi],
+                                     tok["g"][lo:hi], beta=tok["beta"][lo:hi] if tok["beta"] is not None else None,
+                                     u_bonus=rig.bonus[layer], slot_idx=slots_sorted[lo:hi], out=rig.out[lo:hi])
         else:
             (dl.decode_merge_step if t % M == M - 1 else dl.decode_step)(*args, slot_idx=rig.slot_idx, **kw)
 

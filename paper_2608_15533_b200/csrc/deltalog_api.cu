@@ -202,12 +202,12 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     }
     const size_t smem = merge_smem_bytes<D>(st.cap);
     // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
-    // call over a whole batch whose fills are staggered) most units are skipped: eight per CTA.
+    // call over a whole batch whose fills are staggered) most units are skipped: kMergePack candidates per CTA.
     const int pairs = n * st.H;
     if (only_if_full) {
-        auto kernel = merge_kernel<OP, D, IO, UL, 8>;
+        auto kernel = merge_kernel<OP, D, IO, UL, kMergePack>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
-        kernel<<<(pairs + 7) / 8, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
+        kernel<<<(pairs + kMergePack - 1) / kMergePack, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
     } else {
         auto kernel = merge_kernel<OP, D, IO, UL, 1>;
         if (int rc = ensure_smem(kernel, smem)) return rc;

@@ -17,11 +17,17 @@ constexpr size_t merge_smem_bytes(int cap) {
     return sizeof(float) * ((size_t)2 * cap * D + D);  // A [cap][D], U [cap][D] (fp32), e^{lbar} [D]
 }
 
+#ifndef DELTALOG_MERGE_PACK
+#define DELTALOG_MERGE_PACK 16
+#endif
+constexpr int kMergePack = DELTALOG_MERGE_PACK;  // candidates per CTA of a predicate merge
+
 #ifndef DELTALOG_MERGE_CTAS
 #define DELTALOG_MERGE_CTAS 2
 #endif
 // PACK: (listed slot, head) pairs a CTA is responsible for: 1 when every listed unit is expected to
-// fold, 8 for predicate merges over a batch with staggered fills, where most pairs are skipped.
+// fold, kMergePack (strided over the grid) for predicate merges over a batch with staggered fills, where most
+// pairs are skipped.
 template <int OP, int D, typename IO, typename UL, int PACK>
 __global__ void __launch_bounds__(kThreads, DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
@@ -36,7 +42,9 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     __shared__ int s_unit[PACK], s_len[PACK];
     if (PACK > 1) {
         if (tid < PACK) {
-            const int pair = blockIdx.x * PACK + tid;
+            // candidates are strided over the grid: the heads of a full row are consecutive pairs, and
+            // this way they land in different CTAs instead of queueing up in one
+            const int pair = blockIdx.x + tid * gridDim.x;
             int len = 0, unit = 0;
             if (pair < n_pairs) {
                 int slot;
