@@ -131,9 +131,14 @@ class Rig:
         self.out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
         self.slot_idx = None
         self.staggered = bool(wl.staggered)
+        self.predicate_merge = False   # staggered batches: one predicate merge over the whole batch instead of listed rows
+        self.phase = 0
         if self.staggered:  # serving shape: rows address a shuffled slot pool, every row at its own log fill
             self.slot_idx = workloads.slot_permutation(wl).to(device)
             self.delay = ((cap - workloads.fill_offsets(wl, cap)) % cap).to(device)
+            # the host knows every row's phase from its step counter: before step t the rows with
+            # delay == t mod cap hold a full log; their slots, listed per residue, are what the merge gets
+            self.full_slots = [self.slot_idx[self.delay == r].contiguous() for r in range(cap)]
 
     def decode(self, t, layer=0, slot_idx=None):
         tok = self.rings[layer][t % self.RING]
@@ -152,13 +157,28 @@ class Rig:
         self.dl.merge(self.desc, self.states[layer], slot_idx=self.slot_idx, n=self.wl.batch,
                       only_if_full=only_if_full)
 
+    def stag_merge(self, layer=0):
+        """Staggered batch, before a decode step: fold the rows whose log is full -- listed by the host,
+        which knows every row's phase (``self.phase`` = steps since the fills were laid out, mod cap),
+        or found by the predicate merge over the whole batch."""
+        if self.predicate_merge:
+            return self.merge(layer, only_if_full=True)
+        slots = self.full_slots[self.phase]
+        if slots.numel():
+            self.dl.merge(self.desc, self.states[layer], slot_idx=slots, n=slots.numel(), only_if_full=False)
+
+    def end_layer(self, layer):
+        if self.staggered and layer == self.layers - 1:
+            self.phase = (self.phase + 1) % self.cap
+
     def step(self, t, layer=0):
         """One step of the hot path for one layer.  Uniform batch: decode, and the merge after every
-        cap-th step.  Staggered batch: a predicate merge over the whole batch (only full logs fold,
-        about 1/cap of the rows per step), then decode."""
+        cap-th step.  Staggered batch: a merge of the rows whose log is full (about 1/cap of the rows per
+        step), then decode."""
         if self.staggered:
-            self.merge(layer, only_if_full=True)
+            self.stag_merge(layer)
             self.decode(t, layer)
+            self.end_layer(layer)
         else:
             self.decode(t, layer)
             if (t + 1) % self.cap == 0:
@@ -175,6 +195,7 @@ class Rig:
                 slots = torch.where(self.delay <= t, self.slot_idx, torch.full_like(self.slot_idx, -1))
                 for layer in range(self.layers):
                     self.decode(t, layer, slot_idx=slots)
+        self.phase = 0   # before the next step exactly the rows with delay 0 hold a full log
 
     def status(self):
         return [int(s.status.item()) for s in self.states]
@@ -198,10 +219,11 @@ def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
                 if per_kernel and layer == 0:  # one layer in `layers` carries the events
                     marks.append([ev(), ev(), ev()])
                     marks[-1][1].record()       # merge first here: [1] -> merge -> [2]=[0] -> decode -> end
-                    rig.merge(layer, only_if_full=True)
+                    rig.stag_merge(layer)
                     marks[-1][0].record()
                     rig.decode(t, layer)
                     marks[-1][2].record()
+                    rig.end_layer(layer)
                 else:
                     rig.step(t, layer)
                 continue
@@ -230,11 +252,11 @@ def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
 
 
 def graph_steps(cap: int, staggered: bool = False) -> int:
-    """Steps per captured graph: whole cycles that also return to the start of the token ring (a
-    staggered batch launches the same two kernels every step, so the ring length is enough)."""
+    """Steps per captured graph: whole cycles that also return to the start of the token ring (in a
+    staggered batch the list of rows to fold repeats with period cap as well)."""
     import math
 
-    return Rig.RING if staggered else cap * Rig.RING // math.gcd(cap, Rig.RING)
+    return cap * Rig.RING // math.gcd(cap, Rig.RING)
 
 
 def time_graph_loop(rig: Rig, steps: int):
@@ -251,8 +273,7 @@ def time_graph_loop(rig: Rig, steps: int):
             for t in range(g_len):
                 for layer in range(rig.layers):
                     rig.step(t, layer)
-        for _ in range(2 if rig.staggered else 1):  # warm the replay path; an unstaggered graph ends on empty logs,
-            graph.replay()                         # a staggered batch of ring-length graphs needs cap steps per period
+        graph.replay()  # warm the replay path; a graph holds whole cycles, so every replay starts in the same phase
     torch.cuda.synchronize()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launch.barrier()
@@ -561,7 +582,7 @@ def main():
         "config": {
             "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
             "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
-            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("predicate merge over the batch before every step, fills staggered over 0..cap-1" if stag
+            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1" if stag
                       else f"after every {cap}th step"),
             "launch": (f"one CUDA graph of {g_len} steps, replayed" if use_graph else "plain launches"),
             "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
