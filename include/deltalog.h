@@ -79,6 +79,9 @@ typedef struct {
     int32_t klog_dtype; /* deltalog_dtype of K_log */
     int32_t ulog_dtype; /* deltalog_dtype of U_log */
     float scale;        /* multiplies the output of GDN / KDA (ignored for RWKV6) */
+    int32_t H_qk;       /* query/key heads: 0 or H = one per state head; otherwise a divisor of H, and state
+                           head h uses the q and k of head h / (H / H_qk) (grouped heads: several value
+                           heads share one query/key head); q and k are then [B, H_qk, d_k] */
 } deltalog_desc;
 
 /* Physical state (Section 3.1).  Device pointers, caller-owned. d_lambda = 1 (GDN) or d_k. */
@@ -98,6 +101,7 @@ typedef struct {
  * as entry log_len and increments log_len.  Never writes S_base.
  *
  *   q, k, v  [B, H, d]  io_dtype (q is the receptance r for RWKV6)
+ *   q, k     [B, H_qk, d_k] io_dtype (H_qk = H unless the descriptor groups heads); v [B, H, d_v]
  *   g        log-decay lambda_t <= 0, fp32: [B, H] for GDN / RetNet, [B, H, d_k] for KDA / RWKV6 / GLA;
  *            ignored (may be NULL) for plain linear attention
  *   beta     [B, H] fp32 for GDN / KDA; ignored (may be NULL) otherwise

@@ -43,7 +43,7 @@ class DeltalogError(RuntimeError):
 class _Desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("op", "num_slots", "H", "d_k", "d_v", "cap", "io_dtype", "klog_dtype", "ulog_dtype")] + \
-               [("scale", ctypes.c_float)]
+               [("scale", ctypes.c_float), ("H_qk", ctypes.c_int32)]
 
 
 class _State(ctypes.Structure):
@@ -125,6 +125,7 @@ class Desc:
     klog_dtype: Optional[int] = None   # default: io_dtype
     ulog_dtype: Optional[int] = None   # default: F32 for GDN / KDA, io_dtype where b = v
     scale: float = 1.0
+    H_qk: int = 0                      # query/key heads (0 = H); a divisor of H groups value heads
 
     def __post_init__(self):
         if self.klog_dtype is None:
@@ -138,7 +139,7 @@ class Desc:
 
     def c_struct(self) -> _Desc:
         key = (self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
-               self.klog_dtype, self.ulog_dtype, float(self.scale))
+               self.klog_dtype, self.ulog_dtype, float(self.scale), int(self.H_qk))
         cached = self.__dict__.get("_c")
         if cached is None or cached[0] != key:
             cached = (key, _Desc(*key))
@@ -262,7 +263,7 @@ class HostStaging:
 
     def __init__(self, desc: Desc, B: int, device):
         io = _DT_TO_TORCH[desc.io_dtype]
-        self.q = torch.empty(B, desc.H, desc.d_k, dtype=io, device=device)
+        self.q = torch.empty(B, desc.H_qk or desc.H, desc.d_k, dtype=io, device=device)
         self.k = torch.empty_like(self.q)
         self.v = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
         gshape = (B, desc.H, desc.d_k) if desc.op in _VEC_DECAY else (B, desc.H)

@@ -168,6 +168,10 @@ struct TokenArgs {
     const int32_t *slot_idx;
     void *out;
     int32_t B;
+    int32_t H_qk;      // query/key heads
+    int32_t qk_group;  // state heads per query/key head (H / H_qk)
+    // row of q / k that (batch row b, state head h) reads
+    __device__ __forceinline__ size_t qk_row(int b, int h) const { return (size_t)b * H_qk + h / qk_group; }
 };
 
 struct StateArgs {

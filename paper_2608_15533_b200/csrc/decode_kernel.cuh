@@ -102,8 +102,8 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     cp_async_commit();
     if (!kVecDecay && tid < len) Lam_s[tid] = Lg[tid];
 
-    const IO *qg = static_cast<const IO *>(tk.q) + row * D;
-    const IO *kg = static_cast<const IO *>(tk.k) + row * D;
+    const IO *qg = static_cast<const IO *>(tk.q) + tk.qk_row(b, h) * D;
+    const IO *kg = static_cast<const IO *>(tk.k) + tk.qk_row(b, h) * D;
     const IO *vg = static_cast<const IO *>(tk.v) + row * D;
     const float *gg = tk.g + row * DL;
     IO k_raw = from_f32<IO>(0.f);

@@ -324,8 +324,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                                            (OP == DELTALOG_RWKV6 ? D * 4 : 0);
                     mbar_arrive_expect_tx(fa, bytes);
                     const uint32_t sa = smem_addr(stage);
-                    bulk_copy_g2s(sa + lay.q, static_cast<const IO *>(tk.q) + (size_t)item * D, io_vec, fa);
-                    bulk_copy_g2s(sa + lay.k, static_cast<const IO *>(tk.k) + (size_t)item * D, io_vec, fa);
+                    const size_t qk = tk.qk_row(item / H, item % H);
+                    bulk_copy_g2s(sa + lay.q, static_cast<const IO *>(tk.q) + qk * D, io_vec, fa);
+                    bulk_copy_g2s(sa + lay.k, static_cast<const IO *>(tk.k) + qk * D, io_vec, fa);
                     if (kVecDecay) bulk_copy_g2s(sa + lay.g, tk.g + (size_t)item * D, D * 4, fa);
                     if (L > 0) {
                         bulk_copy_g2s(sa + lay.L, st.decay_log + unit * cap * DL, lb, fa);

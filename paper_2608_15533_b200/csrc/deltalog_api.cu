@@ -32,6 +32,7 @@ int validate_desc(const deltalog_desc *d) {
     if (!d) return DELTALOG_ERR_INVALID_ARG;
     if (d->op < DELTALOG_GDN || d->op > DELTALOG_GLA) return DELTALOG_ERR_INVALID_ARG;
     if (d->num_slots <= 0 || d->H <= 0) return DELTALOG_ERR_INVALID_ARG;
+    if (d->H_qk < 0 || (d->H_qk > 0 && d->H % d->H_qk != 0)) return DELTALOG_ERR_INVALID_ARG;
     if (d->io_dtype != DELTALOG_F32 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->klog_dtype != DELTALOG_F32 && d->klog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->ulog_dtype != DELTALOG_F32 && d->ulog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
@@ -61,6 +62,14 @@ int validate_token(const deltalog_desc *d, const void *q, const void *k, const v
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (op_has_gate(d->op) && !aligned16(g)))
         return DELTALOG_ERR_INVALID_ARG;
     return DELTALOG_OK;
+}
+
+int qk_heads(const deltalog_desc *d) { return d->H_qk > 0 ? d->H_qk : d->H; }
+
+TokenArgs make_token_args(const deltalog_desc *d, const void *q, const void *k, const void *v, const float *g,
+                          const float *beta, const float *u_bonus, const int32_t *slot_idx, void *out, int32_t B) {
+    // plain linear attention has no gate: the kernels see a null pointer and use lambda = 0
+    return TokenArgs{q, k, v, op_has_gate(d->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B, qk_heads(d), d->H / qk_heads(d)};
 }
 
 StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
@@ -271,7 +280,7 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
-    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_DECODE(OP, D, IO) return launch_decode<OP, D, IO>(st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
@@ -288,7 +297,7 @@ int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
-    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_FUSED(OP, D, IO) return launch_fused_step<OP, D, IO>(st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_FUSED);
@@ -332,7 +341,7 @@ int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, cons
     if (!S || !aligned16(S)) return DELTALOG_ERR_INVALID_ARG;
     if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
     if (B == 0) return DELTALOG_OK;
-    const TokenArgs tk{q, k, v, op_has_gate(desc->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B};
+    const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 #define CALL_EAGER(OP, D, IO) return launch_eager<OP, D, IO>(S, desc, status, tk, s)
     DELTALOG_DISPATCH(desc, CALL_EAGER);
@@ -354,11 +363,12 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t units = (size_t)B * desc->H;
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
-    const size_t vec = units * desc->d_k * esz;
+    const size_t vec = units * desc->d_v * esz;
+    const size_t qk_vec = (size_t)B * qk_heads(desc) * desc->d_k * esz;
     const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
     if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
-    bool ok = cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    bool ok = cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
     if (op_has_gate(desc->op))
         ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
@@ -395,12 +405,13 @@ int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltal
     cudaEvent_t e_out = static_cast<cudaEvent_t>(lane->out_done);
     const size_t units = (size_t)B * desc->H;
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
-    const size_t vec = units * desc->d_k * esz;
+    const size_t vec = units * desc->d_v * esz;
+    const size_t qk_vec = (size_t)B * qk_heads(desc) * desc->d_k * esz;
     const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
     // copy-in stream: the staging inputs are free once the kernel that last read them is done
     bool ok = cudaStreamWaitEvent(s_in, e_cmp, 0) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->q, host_q, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->k, host_k, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+    ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
     if (op_has_gate(desc->op))
         ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;

@@ -38,8 +38,8 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
 
     const IO *vg = static_cast<const IO *>(tk.v) + row * D;
     if (tid < D) {
-        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[row * D + tid]);
-        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[row * D + tid]);
+        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * D + tid]);
+        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * D + tid]);
         a_s[tid] = tk.g ? expf(tk.g[row * DL + (kVecDecay ? tid : 0)]) : 1.f;  // no gate: plain linear attention
     }
     __syncthreads();

@@ -87,8 +87,8 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     if (tid < D) {
         const int jl = kVecDecay ? tid : 0;
         const float lo = len > 0 ? lold[jl] : 0.f, lam = tk.g ? gg[jl] : 0.f;
-        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[row * D + tid]);
-        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[row * D + tid]);
+        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * D + tid]);
+        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * D + tid]);
         e_s[tid] = expf(kPost ? lo + lam : lo);
         w_s[tid] = expf(lam);
     }
