@@ -105,9 +105,9 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def unit_shape(wl: workloads.Workload) -> traffic.UnitShape:
+def unit_shape(wl: workloads.Workload, ulog16: bool = False) -> traffic.UnitShape:
     io = 4 if wl.io_dtype == torch.float32 else 2
-    ul = io if wl.op == workloads.RWKV6 else 4
+    ul = 4 if wl.op in (workloads.GDN, workloads.KDA) and not ulog16 else io  # b = v keeps the I/O dtype
     return traffic.UnitShape(wl.op, wl.d, wl.d, io_bytes=io, klog_bytes=io, ulog_bytes=ul)
 
 
@@ -116,12 +116,13 @@ class Rig:
 
     RING = 8
 
-    def __init__(self, wl, cap, device, seed_offset=0, layers=1):
+    def __init__(self, wl, cap, device, seed_offset=0, layers=1, ulog16=False):
         import paper_2608_15533_b200 as dl
 
         self.dl, self.wl, self.cap, self.device, self.layers = dl, wl, cap, device, layers
         io = dl.F32 if wl.io_dtype == torch.float32 else dl.BF16
-        self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io)
+        self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
+                            ulog_dtype=io if ulog16 else None)
         self.states, self.rings, self.bonus = [], [], []
         for layer in range(layers):
             src = workloads.TokenSource(wl, device=device, seed=wl.seed + 1000 * seed_offset + layer)

@@ -151,15 +151,33 @@ def study_ablation(steps: int) -> dict:
     return {"study": "ablation", "workload": workloads.CONFIGS[1].name, "cap": 16, "rows": rows}
 
 
+def study_precision(device, steps: int) -> dict:
+    """The value-side log of the delta rule in fp32 (default; meets the 1e-4 state bar) against the
+    16-bit variant (does not: see tests/test_ulog_precision.py): what the smaller entries buy."""
+    wl = workloads.CONFIGS[1]
+    rows = []
+    for name, u16 in (("U log fp32 (default)", False), ("U log bf16 (reduced precision)", True)):
+        rig = bench.Rig(wl, 16, device, ulog16=u16)
+        ms = _split_cycle_ms(rig, steps)
+        assert all(s == 0 for s in rig.status())
+        u = bench.unit_shape(wl, ulog16=u16)
+        cyc = traffic.cycle_bytes(u, 16)
+        rows.append({"variant": name, "entry_bytes": u.entry, "us_per_step": ms * 1e3,
+                     "bytes_per_unit_step": cyc["total"], "hbm_gbs": cyc["total"] * wl.units / (ms * 1e-3) / 1e9})
+        del rig
+        torch.cuda.empty_cache()
+    return {"study": "precision", "workload": wl.name, "cap": 16, "rows": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--study", default="all", choices=["m_sweep", "state_size", "phases", "ablation", "all"])
+    ap.add_argument("--study", default="all", choices=["m_sweep", "state_size", "phases", "ablation", "precision", "all"])
     ap.add_argument("--steps", type=int, default=1024)
     args = ap.parse_args()
     assert torch.cuda.is_available(), "the studies need a CUDA device (there is no CPU path)"
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
-    todo = ["m_sweep", "state_size", "phases", "ablation"] if args.study == "all" else [args.study]
+    todo = ["m_sweep", "state_size", "phases", "ablation", "precision"] if args.study == "all" else [args.study]
     for name in todo:
         if name == "m_sweep":
             res = study_m_sweep(device, args.steps)
@@ -167,6 +185,8 @@ def main():
             res = study_state_size(device, args.steps)
         elif name == "phases":
             res = study_phases(device, args.steps)
+        elif name == "precision":
+            res = study_precision(device, args.steps)
         else:
             res = study_ablation(args.steps)
         print(json.dumps(res), flush=True)

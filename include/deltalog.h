@@ -35,7 +35,9 @@
  *     on; kernels never trap.  Rows with slot index < 0 are padding and are skipped silently.
  *   - The same slot must not appear twice in one call.
  *   - Supported shapes: d_k == d_v in {64, 128}; 1 <= cap <= 64; klog_dtype == io_dtype;
- *     ulog_dtype == F32 for GDN / KDA and == io_dtype for the operators with b_t = v_t.
+ *     ulog_dtype == io_dtype for the operators with b_t = v_t; F32 for GDN / KDA (the paper keeps b_t in
+ *     fp32 against cancellation in the correction path), or, as a reduced-precision variant that does
+ *     NOT meet the 1e-4 state tolerance, == io_dtype == BF16.
  */
 #ifndef DELTALOG_H
 #define DELTALOG_H

@@ -27,8 +27,11 @@ ADDITIVE = (LINATTN, RETNET, GLA)  # b = v, readout from the updated state; LINA
 class LogState:
     """Base + bounded log for ``N`` independent (sequence, head) units (Section 3.1)."""
 
-    def __init__(self, op: int, S0: np.ndarray, cap: int):
+    def __init__(self, op: int, S0: np.ndarray, cap: int, store_u=None):
+        """``store_u``: optional function applied to a value-side factor when it is written into the
+        log (e.g. rounding to a 16-bit format), for studies of reduced-precision logs; None = exact."""
         S0 = np.asarray(S0, dtype=np.float64)
+        self.store_u = store_u
         self.op = int(op)
         self.N, self.d_k, self.d_v = S0.shape
         self.cap = int(cap)
@@ -103,7 +106,7 @@ def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float 
             b = float(beta[n]) * (v[n] - S_decayed.T @ k[n])
         # lines 4-5 / Eq. 4: append (a, b, lbar) into slot L; the base is untouched
         st.K_log[n, L] = a
-        st.U_log[n, L] = b
+        st.U_log[n, L] = b if st.store_u is None else st.store_u(b)
         st.Lam_log[n, L] = st.lbar[n]
         st.length[n] = L + 1
         if st.op != RWKV6:

@@ -38,8 +38,11 @@ int validate_desc(const deltalog_desc *d) {
     if (d->ulog_dtype != DELTALOG_F32 && d->ulog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
     if (d->d_k != d->d_v || (d->d_k != 64 && d->d_k != 128)) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     if (d->klog_dtype != d->io_dtype) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    const int want_u = op_delta_rule(d->op) ? (int)DELTALOG_F32 : d->io_dtype;  // b = v is lossless in the I/O dtype
-    if (d->ulog_dtype != want_u) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
+    // b = v is lossless in the I/O dtype; the delta rule keeps b in fp32 unless the caller asks for the
+    // reduced-precision 16-bit U log (only with 16-bit I/O)
+    const bool u_ok = op_delta_rule(d->op) ? (d->ulog_dtype == DELTALOG_F32 || d->ulog_dtype == d->io_dtype)
+                                           : d->ulog_dtype == d->io_dtype;
+    if (!u_ok) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     if (d->cap < 1 || d->cap > kMaxCap) return DELTALOG_ERR_CAP_RANGE;
     return DELTALOG_OK;
 }
@@ -140,9 +143,8 @@ int env_int(const char *name, int dflt) {
     return v ? std::atoi(v) : dflt;
 }
 
-template <int OP, int D, typename IO>
+template <int OP, int D, typename IO, typename UL>
 int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
     static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
     static const int env_base = env_int("DELTALOG_BASE_STAGES", 0);
@@ -189,10 +191,9 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
     return finish_launch();
 }
 
-template <int OP, int D, typename IO>
+template <int OP, int D, typename IO, typename UL>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
-    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     // DELTALOG_MERGE_TC = 1 (head size 128, no predicate): the contraction over the log entries runs
     // on the tensor cores (tcgen05, tf32 x 3).  Off by default: it executes a fraction of the
     // instructions, but with one unit per CTA the extra hand-overs (raw entries -> operands -> MMA ->
@@ -225,9 +226,8 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     return finish_launch();
 }
 
-template <int OP, int D, typename IO>
+template <int OP, int D, typename IO, typename UL>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    using UL = typename std::conditional<OpTraits<OP>::kDeltaRule, float, IO>::type;
     auto kernel = decode_merge_step_kernel<OP, D, IO, UL>;
     const size_t smem = fused_step_smem_bytes<D>(st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
@@ -264,6 +264,20 @@ int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenA
         if (io_ == DELTALOG_F32) { CALL(OP, 128, float); } else { CALL(OP, 128, __nv_bfloat16); } \
     }
 
+// The value-side log keeps the I/O dtype where b = v (lossless).  For the delta rule it is fp32 by
+// default; a 16-bit U log (descriptor ulog_dtype == io_dtype == BF16) is the reduced-precision variant.
+#define DELTALOG_WITH_UL(OP, IO, desc, FN, D, ...)                                                         \
+    do {                                                                                                  \
+        if constexpr (OpTraits<OP>::kDeltaRule) {                                                         \
+            if constexpr (!std::is_same<IO, float>::value) {                                              \
+                if ((desc)->ulog_dtype != DELTALOG_F32) return FN<OP, D, IO, IO>(__VA_ARGS__);             \
+            }                                                                                             \
+            return FN<OP, D, IO, float>(__VA_ARGS__);                                                     \
+        } else {                                                                                          \
+            return FN<OP, D, IO, IO>(__VA_ARGS__);                                                        \
+        }                                                                                                 \
+    } while (0)
+
 }  // namespace
 }  // namespace deltalog
 
@@ -282,7 +296,7 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
     const StateArgs st = make_state_args(desc, state);
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_DECODE(OP, D, IO) return launch_decode<OP, D, IO>(st, tk, s)
+#define CALL_DECODE(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode, D, st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
 #undef CALL_DECODE
     return DELTALOG_ERR_INVALID_ARG;
@@ -299,7 +313,7 @@ int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *
     const StateArgs st = make_state_args(desc, state);
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_FUSED(OP, D, IO) return launch_fused_step<OP, D, IO>(st, tk, s)
+#define CALL_FUSED(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_fused_step, D, st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_FUSED);
 #undef CALL_FUSED
     return DELTALOG_ERR_INVALID_ARG;
@@ -313,7 +327,7 @@ int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const
     if (n == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_MERGE(OP, D, IO) return launch_merge<OP, D, IO>(st, slot_idx, n, only_if_full, s)
+#define CALL_MERGE(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_merge, D, st, slot_idx, n, only_if_full, s)
     DELTALOG_DISPATCH(desc, CALL_MERGE);
 #undef CALL_MERGE
     return DELTALOG_ERR_INVALID_ARG;

@@ -59,7 +59,9 @@ def test_host_side_rejections_launch_nothing(lib):
     assert _decode(lib, _desc(d_k=64, d_v=128), s) == binding.ERR_UNSUPPORTED_SHAPE
     assert _decode(lib, _desc(cap=0), s) == binding.ERR_CAP_RANGE
     assert _decode(lib, _desc(cap=65), s) == binding.ERR_CAP_RANGE
-    assert _decode(lib, _desc(ulog_dtype=dl.BF16), s) == binding.ERR_UNSUPPORTED_SHAPE     # delta rule keeps U in fp32
+    # a 16-bit U log for the delta rule needs 16-bit I/O; where b = v the U log has the I/O dtype
+    assert _decode(lib, _desc(io_dtype=dl.F32, klog_dtype=dl.F32, ulog_dtype=dl.BF16), s) == binding.ERR_UNSUPPORTED_SHAPE
+    assert _decode(lib, _desc(op=dl.RWKV6, ulog_dtype=dl.F32), s, bonus=0x70000) == binding.ERR_UNSUPPORTED_SHAPE
     assert _decode(lib, _desc(klog_dtype=dl.F32), s) == binding.ERR_UNSUPPORTED_SHAPE
     assert _decode(lib, _desc(num_slots=0), s) == binding.ERR_INVALID_ARG
     assert _decode(lib, _desc(), _state(null="S_base")) == binding.ERR_INVALID_ARG
