@@ -3,7 +3,7 @@
 sweep with the U-shaped latency curve, state-size scaling, the split-preparation ablation and the
 per-phase costs).  Synthetic inputs of configuration 1's shape (GDN, H = 32, d = 128, bf16 I/O).
 
-    python bench_studies.py [--study m_sweep|state_size|phases|ablation|all] [--steps K]
+    python bench_studies.py [--study m_sweep|state_size|phases|ablation|precision|multi_token|all] [--steps K]
 
 Prints one JSON object per study.  Everything is timed with CUDA events on the launch stream after
 warm-up; cycles are replayed from CUDA graphs exactly as in bench.py, whose rig this script reuses.
@@ -169,15 +169,73 @@ def study_precision(device, steps: int) -> dict:
     return {"study": "precision", "workload": wl.name, "cap": 16, "rows": rows}
 
 
+def study_multi_token(device, steps: int) -> dict:
+    """Blocks of T tokens per call (deltalog_decode_steps: one read of the base tile per block) against
+    single-token steps, on configuration 1's shape at cap 16: a cycle is 16 / T block calls and the
+    merge, replayed from a CUDA graph.  Per-token cost and algorithmic bytes."""
+    import paper_2608_15533_b200 as dl
+
+    wl, cap = workloads.CONFIGS[1], 16
+    rig = bench.Rig(wl, cap, device)
+    u = bench.unit_shape(wl)
+    rows = []
+    for T in (1, 2, 4, 8, 16):
+        blocks = [{k: (torch.stack([rig.rings[0][(i * T + t) % rig.RING][k] for t in range(T)], dim=1).contiguous()
+                       if rig.rings[0][0][k] is not None else None) for k in rig.rings[0][0]}
+                  for i in range(rig.RING)]
+        out = torch.empty(wl.batch, T, wl.H, wl.d, dtype=wl.io_dtype, device=device)
+        rig.reset_logs()
+
+        def cycle(i0):
+            for i in range(cap // T):
+                tok = blocks[(i0 + i) % rig.RING]
+                dl.decode_steps(rig.desc, rig.states[0], tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                                out=out)
+            rig.merge()
+
+        cycle(0)
+        stream = torch.cuda.Stream(device=device)
+        graph = torch.cuda.CUDAGraph()
+        torch.cuda.synchronize()
+        n_cycles_graph = 8
+        with torch.cuda.stream(stream):
+            with torch.cuda.graph(graph, stream=stream):
+                for c in range(n_cycles_graph):
+                    cycle(c)
+            graph.replay()
+        torch.cuda.synchronize()
+        reps = max(steps // (cap * n_cycles_graph), 1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            a.record()
+            for _ in range(reps):
+                graph.replay()
+            b.record()
+        torch.cuda.synchronize()
+        assert all(s == 0 for s in rig.status())
+        us_per_token = a.elapsed_time(b) * 1e3 / (reps * n_cycles_graph * cap)
+        # bytes per unit and token: one base read per block, the live log once per block, token I/O and appends per token
+        blocks_per_cycle = cap // T
+        rd = sum(u.state + (i * T) * u.entry + traffic.LEN_WORD for i in range(blocks_per_cycle)) + cap * u.token_in
+        wr = cap * (u.entry + u.token_out) + blocks_per_cycle * traffic.LEN_WORD
+        total = rd + wr + traffic.merge_read(u, cap) + traffic.merge_write(u)
+        rows.append({"T": T, "us_per_token": us_per_token, "bytes_per_unit_token": total / cap,
+                     "hbm_gbs": total / cap * wl.units / (us_per_token * 1e-6) / 1e9,
+                     "kernel": "one CTA per unit, tile in registers"})
+    return {"study": "multi_token", "workload": wl.name, "cap": cap,
+            "note": "T = 1 through deltalog_decode_steps uses the one-CTA-per-unit kernel; the single-token entry point "
+                    "(persistent kernel) runs the same cycle at the figure bench.py reports", "rows": rows}
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--study", default="all", choices=["m_sweep", "state_size", "phases", "ablation", "precision", "all"])
+    ap.add_argument("--study", default="all", choices=["m_sweep", "state_size", "phases", "ablation", "precision", "multi_token", "all"])
     ap.add_argument("--steps", type=int, default=1024)
     args = ap.parse_args()
     assert torch.cuda.is_available(), "the studies need a CUDA device (there is no CPU path)"
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
-    todo = ["m_sweep", "state_size", "phases", "ablation", "precision"] if args.study == "all" else [args.study]
+    todo = ["m_sweep", "state_size", "phases", "ablation", "precision", "multi_token"] if args.study == "all" else [args.study]
     for name in todo:
         if name == "m_sweep":
             res = study_m_sweep(device, args.steps)
@@ -187,6 +245,8 @@ def main():
             res = study_phases(device, args.steps)
         elif name == "precision":
             res = study_precision(device, args.steps)
+        elif name == "multi_token":
+            res = study_multi_token(device, args.steps)
         else:
             res = study_ablation(args.steps)
         print(json.dumps(res), flush=True)

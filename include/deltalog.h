@@ -117,6 +117,20 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
                          void *stream);
 
 /*
+ * T consecutive tokens for each of the B rows in one call (several tokens of a request at once, e.g.
+ * the verification step of speculative decoding).  Results are those of T successive
+ * deltalog_decode_step calls; the base tile is read once for all T tokens.  Token tensors carry a
+ * token axis after the batch axis: q, k [B, T, H_qk, d_k]; v, out [B, T, H, d_v]; g [B, T, H] or
+ * [B, T, H, d_k]; beta [B, T, H].  1 <= T <= cap (DELTALOG_ERR_CAP_RANGE otherwise).  A (row, head)
+ * whose log has no room for all T entries (log_len + T > cap) is skipped as a whole -- nothing is
+ * appended, `out` is not written -- and DELTALOG_STATUS_LOG_FULL is raised.  The paper's decode path
+ * is single-token; this entry point extends its append branch (Algorithm 1) to a block of tokens.
+ */
+int deltalog_decode_steps(const deltalog_desc *desc, const deltalog_state *state, const void *q, const void *k,
+                          const void *v, const float *g, const float *beta, const float *u_bonus,
+                          const int32_t *slot_idx, int32_t B, int32_t T, void *out, void *stream);
+
+/*
  * The merge step of the cycle as the paper runs it (Algorithm 1, else-branch; Eq. 5 with the
  * current-token term): every row of the batch consumes its token AND has its state materialised,
  *     lbar <- lbar + lambda_t ;  (a_t, b_t) and `out` exactly as in deltalog_decode_step ;

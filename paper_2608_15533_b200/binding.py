@@ -28,7 +28,7 @@ _DT_TO_TORCH = {F32: torch.float32, BF16: torch.bfloat16}
 LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
 
 EXPORTS = (
-    "deltalog_decode_step", "deltalog_decode_merge_step", "deltalog_merge", "deltalog_reset_slots", "deltalog_eager_step", "deltalog_decode_step_host",
+    "deltalog_decode_step", "deltalog_decode_steps", "deltalog_decode_merge_step", "deltalog_merge", "deltalog_reset_slots", "deltalog_eager_step", "deltalog_decode_step_host",
     "deltalog_decode_step_host_static", "deltalog_decode_step_host_overlapped",
     "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
 )
@@ -74,6 +74,8 @@ def load_library() -> ctypes.CDLL:
         vp, i32 = ctypes.c_void_p, ctypes.c_int32
         lib.deltalog_decode_step.restype = ctypes.c_int
         lib.deltalog_decode_step.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State)] + [vp] * 7 + [i32, vp, vp]
+        lib.deltalog_decode_steps.restype = ctypes.c_int
+        lib.deltalog_decode_steps.argtypes = [ctypes.POINTER(_Desc), ctypes.POINTER(_State)] + [vp] * 7 + [i32, i32, vp, vp]
         lib.deltalog_decode_merge_step.restype = ctypes.c_int
         lib.deltalog_decode_merge_step.argtypes = lib.deltalog_decode_step.argtypes
         lib.deltalog_merge.restype = ctypes.c_int
@@ -204,6 +206,21 @@ def decode_step(desc: Desc, state: State, q, k, v, g, beta=None, u_bonus=None, s
         ctypes.byref(d), ctypes.byref(s), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(u_bonus),
         _ptr(slot_idx), B, _ptr(out), _stream(stream))
     _check(rc, "deltalog_decode_step")
+    return out
+
+
+def decode_steps(desc: Desc, state: State, q, k, v, g, beta=None, u_bonus=None, slot_idx=None, out=None,
+                 stream=None) -> torch.Tensor:
+    """``deltalog_decode_steps``: ``T = q.shape[1]`` consecutive tokens per row (token tensors
+    ``[B,T,H,d]``) with one read of the base tile; returns ``out [B,T,H,d_v]``."""
+    B, T = q.shape[0], q.shape[1]
+    if out is None:
+        out = torch.empty(B, T, desc.H, desc.d_v, dtype=q.dtype, device=q.device)
+    d, s = desc.c_struct(), state.c_struct()
+    rc = load_library().deltalog_decode_steps(
+        ctypes.byref(d), ctypes.byref(s), _ptr(q), _ptr(k), _ptr(v), _ptr(g), _ptr(beta), _ptr(u_bonus),
+        _ptr(slot_idx), B, T, _ptr(out), _stream(stream))
+    _check(rc, "deltalog_decode_steps")
     return out
 
 

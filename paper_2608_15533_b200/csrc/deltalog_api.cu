@@ -10,6 +10,7 @@
 #include <cstdlib>
 
 #include "decode_kernel.cuh"
+#include "decode_multi_kernel.cuh"
 #include "decode_pipelined.cuh"
 #include "eager_kernel.cuh"
 #include "fused_step_kernel.cuh"
@@ -192,6 +193,15 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
 }
 
 template <int OP, int D, typename IO, typename UL>
+int launch_decode_multi(const StateArgs &st, const TokenArgs &tk, int32_t T, cudaStream_t stream) {
+    auto kernel = decode_multi_kernel<OP, D, IO, UL>;
+    const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
+    if (int rc = ensure_smem(kernel, smem)) return rc;
+    kernel<<<tk.B * st.H, decode_threads<D>(), smem, stream>>>(st, tk, T);
+    return finish_launch();
+}
+
+template <int OP, int D, typename IO, typename UL>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
     // DELTALOG_MERGE_TC = 1 (head size 128, no predicate): the contraction over the log entries runs
@@ -299,6 +309,23 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
 #define CALL_DECODE(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode, D, st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
 #undef CALL_DECODE
+    return DELTALOG_ERR_INVALID_ARG;
+}
+
+int deltalog_decode_steps(const deltalog_desc *desc, const deltalog_state *state, const void *q, const void *k,
+                          const void *v, const float *g, const float *beta, const float *u_bonus,
+                          const int32_t *slot_idx, int32_t B, int32_t T, void *out, void *stream) {
+    if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
+    if (int rc = validate_token(desc, q, k, v, g, beta, u_bonus, B, out)) return rc;
+    if (T < 1 || T > desc->cap) return DELTALOG_ERR_CAP_RANGE;
+    if (B == 0) return DELTALOG_OK;
+    const StateArgs st = make_state_args(desc, state);
+    const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+#define CALL_MULTI(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode_multi, D, st, tk, T, s)
+    DELTALOG_DISPATCH(desc, CALL_MULTI);
+#undef CALL_MULTI
     return DELTALOG_ERR_INVALID_ARG;
 }
 
