@@ -123,6 +123,11 @@ class Rig:
         io = dl.F32 if wl.io_dtype == torch.float32 else dl.BF16
         self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
                             ulog_dtype=io if ulog16 else None)
+        # the same problem with the promise that the launch in front of a decode step leaves the base
+        # alone (true for every decode step of a cycle but the first after a merge)
+        self.desc_chained = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
+                                    ulog_dtype=io if ulog16 else None, hints=dl.HINT_BASE_UNTOUCHED)
+        self.chain = os.environ.get("DELTALOG_BENCH_CHAIN", "1") != "0"
         self.states, self.rings, self.bonus = [], [], []
         for layer in range(layers):
             src = workloads.TokenSource(wl, device=device, seed=wl.seed + 1000 * seed_offset + layer)
@@ -141,9 +146,10 @@ class Rig:
             # delay == t mod cap hold a full log; their slots, listed per residue, are what the merge gets
             self.full_slots = [self.slot_idx[self.delay == r].contiguous() for r in range(cap)]
 
-    def decode(self, t, layer=0, slot_idx=None):
+    def decode(self, t, layer=0, slot_idx=None, chained=False):
+        """``chained``: the launch in front of this one on the stream was a decode step of this state."""
         tok = self.rings[layer][t % self.RING]
-        self.dl.decode_step(self.desc, self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
+        self.dl.decode_step(self.desc_chained if (chained and self.chain) else self.desc, self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
                             beta=tok["beta"], u_bonus=self.bonus[layer],
                             slot_idx=self.slot_idx if slot_idx is None else slot_idx, out=self.out)
 
@@ -181,7 +187,7 @@ class Rig:
             self.decode(t, layer)
             self.end_layer(layer)
         else:
-            self.decode(t, layer)
+            self.decode(t, layer, chained=(self.layers == 1 and t % self.cap != 0))
             if (t + 1) % self.cap == 0:
                 self.merge(layer)
 
@@ -231,7 +237,7 @@ def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
             if per_kernel and layer == 0 and t % cap == 0:
                 marks.append([ev(), None, None])
                 marks[-1][0].record()
-            rig.decode(t, layer)
+            rig.decode(t, layer, chained=(rig.layers == 1 and t % cap != 0))
             if (t + 1) % cap == 0:
                 if per_kernel and layer == 0:
                     marks[-1][1] = ev(); marks[-1][1].record()

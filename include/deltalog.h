@@ -84,7 +84,21 @@ typedef struct {
     int32_t H_qk;       /* query/key heads: 0 or H = one per state head; otherwise a divisor of H, and state
                            head h uses the q and k of head h / (H / H_qk) (grouped heads: several value
                            heads share one query/key head); q and k are then [B, H_qk, d_k] */
+    int32_t hints;      /* DELTALOG_HINT_* bits, 0 = none */
 } deltalog_desc;
+
+/*
+ * Hints (deltalog_desc.hints).  A hint is a promise by the caller; breaking it is a data race.
+ *   DELTALOG_HINT_BASE_UNTOUCHED  The work queued on the stream directly in front of this
+ *       deltalog_decode_step does not write S_base of the slots this call reads (it was another
+ *       decode step on this state, or unrelated work -- NOT a deltalog_merge, deltalog_decode_merge_step,
+ *       deltalog_reset_slots or deltalog_eager_step on these slots).  The decode kernel is then
+ *       launched with programmatic stream serialisation: its CTAs start while the preceding kernel is
+ *       still retiring and stream base tiles at once; lengths, log entries and everything else are
+ *       read only after the preceding kernel has completed.  The paper has no counterpart; it removes the
+ *       ramp-up and tail of back-to-back decode launches (a few microseconds each).
+ */
+enum { DELTALOG_HINT_BASE_UNTOUCHED = 1 };
 
 /* Physical state (Section 3.1).  Device pointers, caller-owned. d_lambda = 1 (GDN) or d_k. */
 typedef struct {

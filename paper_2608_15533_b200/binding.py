@@ -15,6 +15,7 @@ from typing import Optional
 import torch
 
 GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+HINT_BASE_UNTOUCHED = 1
 _DELTA_RULE = (GDN, KDA)            # b = beta (v - S'^T k): U log in fp32
 _VEC_DECAY = (KDA, RWKV6, GLA)      # one log-decay per key channel
 F32, BF16 = 0, 1
@@ -43,7 +44,7 @@ class DeltalogError(RuntimeError):
 class _Desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("op", "num_slots", "H", "d_k", "d_v", "cap", "io_dtype", "klog_dtype", "ulog_dtype")] + \
-               [("scale", ctypes.c_float), ("H_qk", ctypes.c_int32)]
+               [("scale", ctypes.c_float), ("H_qk", ctypes.c_int32), ("hints", ctypes.c_int32)]
 
 
 class _State(ctypes.Structure):
@@ -128,6 +129,7 @@ class Desc:
     ulog_dtype: Optional[int] = None   # default: F32 for GDN / KDA, io_dtype where b = v
     scale: float = 1.0
     H_qk: int = 0                      # query/key heads (0 = H); a divisor of H groups value heads
+    hints: int = 0                     # HINT_* bits (promises by the caller, see the header)
 
     def __post_init__(self):
         if self.klog_dtype is None:
@@ -141,7 +143,7 @@ class Desc:
 
     def c_struct(self) -> _Desc:
         key = (self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
-               self.klog_dtype, self.ulog_dtype, float(self.scale), int(self.H_qk))
+               self.klog_dtype, self.ulog_dtype, float(self.scale), int(self.H_qk), int(self.hints))
         cached = self.__dict__.get("_c")
         if cached is None or cached[0] != key:
             cached = (key, _Desc(*key))

@@ -170,6 +170,7 @@ struct TokenArgs {
     int32_t B;
     int32_t H_qk;      // query/key heads
     int32_t qk_group;  // state heads per query/key head (H / H_qk)
+    int32_t hints;     // DELTALOG_HINT_* bits of the descriptor
     // row of q / k that (batch row b, state head h) reads
     __device__ __forceinline__ size_t qk_row(int b, int h) const { return (size_t)b * H_qk + h / qk_group; }
 };

@@ -71,6 +71,12 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 #pragma unroll
     for (int p = 0; p < NP; ++p) s[p] = __ldg(Sg + (size_t)(p * RL + rl) * C4 + c4);
 
+    // Programmatic dependent launch (see DELTALOG_HINT_BASE_UNTOUCHED): the kernel queued behind this
+    // one may start as this one's CTAs retire; and if this kernel itself was started early, everything
+    // the previous step wrote (lengths, log entries) is read only after that step has completed.  The
+    // base tile above was requested before: the caller promised that the previous kernel leaves it alone.
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
     const int len = st.log_len[unit];
     if (len >= cap) {  // Algorithm 1's else-branch is the caller's job (deltalog_merge)
         if (tid == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);

@@ -223,6 +223,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
     __syncthreads();
+    // Programmatic dependent launch: a kernel queued behind this one may start its CTAs as this one's
+    // retire (it synchronises with griddepcontrol.wait before it touches anything written here).
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
     const int total = tk.B * st.H;
     const int first = blockIdx.x, stride = gridDim.x;
@@ -276,6 +279,10 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         bool dead = false;
         long long issued = 0;
         const int io_vec = D * (int)sizeof(IO);
+        // Lengths and log entries are written by the step before this one: when this kernel was
+        // launched ahead of the previous kernel's completion, wait for it here (a no-op otherwise).
+        // Everything the other roles do with global memory follows from what this warp loads.
+        asm volatile("griddepcontrol.wait;\n" ::: "memory");
         for (int it0 = 0; it0 < n_items; it0 += 32) {
             int slot = -1, len = 0, flags = kMetaSkip;
             float gs = 0.f, bt = 0.f;

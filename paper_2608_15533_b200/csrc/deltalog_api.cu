@@ -73,7 +73,8 @@ int qk_heads(const deltalog_desc *d) { return d->H_qk > 0 ? d->H_qk : d->H; }
 TokenArgs make_token_args(const deltalog_desc *d, const void *q, const void *k, const void *v, const float *g,
                           const float *beta, const float *u_bonus, const int32_t *slot_idx, void *out, int32_t B) {
     // plain linear attention has no gate: the kernels see a null pointer and use lambda = 0
-    return TokenArgs{q, k, v, op_has_gate(d->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B, qk_heads(d), d->H / qk_heads(d)};
+    return TokenArgs{q, k, v, op_has_gate(d->op) ? g : nullptr, beta, u_bonus, slot_idx, out, B, qk_heads(d), d->H / qk_heads(d),
+                     d->hints};
 }
 
 StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
@@ -115,6 +116,29 @@ int ensure_smem(K kernel, size_t bytes) {
         return DELTALOG_ERR_CUDA;
     }
     g = bytes;
+    return DELTALOG_OK;
+}
+
+// Launch with programmatic stream serialisation: the caller promised (DELTALOG_HINT_BASE_UNTOUCHED) that
+// the kernel in front of this one on the stream does not write this state's base tiles, so this
+// kernel's CTAs may start, and request base tiles, while that kernel is still retiring.
+template <typename K, typename... Args>
+int launch_chained(K kernel, int grid, int threads, size_t smem, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(grid);
+    lc.blockDim = dim3(threads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (cudaLaunchKernelEx(&lc, kernel, args...) != cudaSuccess) {
+        cudaGetLastError();
+        return DELTALOG_ERR_CUDA;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     return DELTALOG_OK;
 }
 
@@ -182,12 +206,14 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
         const int smem = pipe_smem_bytes<OP, D, IO, UL>(st.cap, cfg);
         if (int rc = ensure_smem(kernel, smem)) return rc;
         const int grid = total < dev.sms * ctas ? total : dev.sms * ctas;
+        if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, grid, kPipeThreads, smem, stream, st, tk, cfg);
         kernel<<<grid, kPipeThreads, smem, stream>>>(st, tk, cfg);
         return finish_launch();
     }
     auto kernel = decode_append_kernel<OP, D, IO, UL>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
+    if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, total, decode_threads<D>(), smem, stream, st, tk);
     kernel<<<total, decode_threads<D>(), smem, stream>>>(st, tk);
     return finish_launch();
 }

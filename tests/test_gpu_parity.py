@@ -380,3 +380,37 @@ def test_predicate_merge_at_capacity_64_head_size_128(op):
     rec, state, S0u, bonus = run_deltalog(wl, 64, DEV, units=[(0, 0), (2, 1), (4, 2)])
     assert 64 in rec.state_at and 128 in rec.state_at
     check_rollout(wl, rec, oracle_for(wl, rec, S0u, bonus))
+
+
+@pytest.mark.parametrize("op,d", [(GDN, 128), (KDA, 128), (RWKV6, 64)])
+def test_chained_launches_are_bit_identical(op, d):
+    """Decode steps that follow a decode step of the same state may be launched ahead of its completion
+    (the caller's hint): lengths and log entries are still read only after it has finished."""
+    import paper_2608_15533_b200 as dl
+
+    wl = small(op, d, torch.bfloat16, batch=40, H=8, steps=48)
+    cap = 16
+    results = []
+    for chained in (False, True):
+        src = workloads.TokenSource(wl, device="cpu")
+        S0 = src.initial_state().to(DEV)
+        bonus = src.bonus()
+        bonus = bonus.to(DEV) if bonus is not None else None
+        toks = [{k_: (v_.to(DEV) if v_ is not None else None) for k_, v_ in src.token().items()} for _ in range(wl.steps)]
+        desc = make_desc(wl, cap)
+        desc_c = make_desc(wl, cap)
+        desc_c.hints = dl.HINT_BASE_UNTOUCHED if chained else 0
+        state = dl.State(desc, S0.clone())
+        outs = [torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=DEV) for _ in range(wl.steps)]
+        torch.cuda.synchronize()
+        for t, tok in enumerate(toks):     # launched back to back, nothing in between
+            first = t % cap == 0
+            if first and t:
+                dl.merge(desc, state)
+            dl.decode_step(desc if first else desc_c, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                           u_bonus=bonus, out=outs[t])
+        dl.merge(desc, state)
+        torch.cuda.synchronize()
+        assert int(state.status.item()) == 0
+        results.append((torch.stack(outs), state.S_base.clone()))
+    assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
