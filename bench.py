@@ -344,8 +344,11 @@ def time_paper_cycle(rig: Rig, steps: int):
                 dl.decode_merge_step(rig.desc, rig.states[layer], tok["q"][lo:hi], tok["k"][lo:hi], tok["v"][lo:hi],
                                      tok["g"][lo:hi], beta=tok["beta"][lo:hi] if tok["beta"] is not None else None,
                                      u_bonus=rig.bonus[layer], slot_idx=slots_sorted[lo:hi], out=rig.out[lo:hi])
-        else:
-            (dl.decode_merge_step if t % M == M - 1 else dl.decode_step)(*args, slot_idx=rig.slot_idx, **kw)
+        elif t % M == M - 1:
+            dl.decode_merge_step(*args, slot_idx=rig.slot_idx, **kw)
+        else:   # every append but the first after the fused step follows a decode step of this state
+            desc = rig.desc_chained if (rig.chain and rig.layers == 1 and t % M != 0) else rig.desc
+            dl.decode_step(desc, *args[1:], slot_idx=rig.slot_idx, **kw)
 
     stream = torch.cuda.Stream(device=rig.device)
     graph = torch.cuda.CUDAGraph()
