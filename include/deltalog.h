@@ -198,12 +198,19 @@ int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, cons
  * staging buffers on `stream`, runs the decode step there and copies `out` back to host_out.
  * The state, u_bonus and slot_idx stay device-resident.  Staging buffers have the shapes of the
  * tensors they stage.  Returns after enqueuing; synchronise the stream before reading host_out.
+ * Packed buffers (staging->packed != 0): q, k, v, g (operators with a gate) and beta (delta rule)
+ * follow one another in this order, each starting on the next 256-byte boundary after the previous
+ * one ends, inside one allocation -- in host memory AND in the staging buffers alike.  The copies then
+ * collapse into one over the whole block (small host-to-device copies run far below the link rate).
+ * If the pointers do not have that layout the flag is ignored and every tensor is copied on its own.
  */
 typedef struct {
     void *q, *k, *v; /* device, [B, H, d] io_dtype */
     float *g;        /* device, shape of g */
     float *beta;     /* device, [B, H]; unused for RWKV6 */
     void *out;       /* device, [B, H, d_v] io_dtype */
+    int32_t packed;  /* != 0: the caller promises that q, k, v, g, beta are carved out of ONE allocation in
+                        the packed layout described below, here and in host memory alike */
 } deltalog_staging;
 
 int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *state,

@@ -52,7 +52,7 @@ class _State(ctypes.Structure):
 
 
 class _Staging(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_void_p) for n in ("q", "k", "v", "g", "beta", "out")]
+    _fields_ = [(n, ctypes.c_void_p) for n in ("q", "k", "v", "g", "beta", "out")] + [("packed", ctypes.c_int32)]
 
 
 class _Lane(ctypes.Structure):
@@ -277,21 +277,53 @@ def eager_step(desc: Desc, S: torch.Tensor, q, k, v, g, beta=None, u_bonus=None,
     return out
 
 
+def _packed_views(desc: "Desc", B: int, block: torch.Tensor):
+    """q, k, v, g, beta as views into one byte block, each starting on the next 256-byte boundary
+    after the previous one ends (the layout the library recognises and copies in one piece)."""
+    io = _DT_TO_TORCH[desc.io_dtype]
+    esz = torch.empty((), dtype=io).element_size()
+    Hqk = desc.H_qk or desc.H
+    gshape = (B, desc.H, desc.d_k) if desc.op in _VEC_DECAY else (B, desc.H)
+    specs = [("q", (B, Hqk, desc.d_k), io), ("k", (B, Hqk, desc.d_k), io), ("v", (B, desc.H, desc.d_v), io),
+             ("g", gshape, torch.float32), ("beta", (B, desc.H), torch.float32)]
+    out, off = {}, 0
+    for name, shape, dt in specs:
+        n = 1
+        for x in shape:
+            n *= x
+        nbytes = n * (esz if dt == io else 4)
+        if block is not None:
+            out[name] = block[off:off + nbytes].view(dt).view(*shape)
+        off = (off + nbytes + 255) // 256 * 256
+    return out, off
+
+
+def packed_host_tokens(desc: "Desc", B: int) -> dict:
+    """Pinned host tensors q, k, v, g, beta laid out back to back (256-byte aligned) in one block:
+    together with ``HostStaging`` the host-buffer entry points then issue a single copy."""
+    _, total = _packed_views(desc, B, None)
+    block = torch.empty(total, dtype=torch.uint8).pin_memory()
+    views, _ = _packed_views(desc, B, block)
+    views["_block"] = block
+    return views
+
+
 class HostStaging:
-    """Device staging buffers for ``decode_step_host`` (allocated once, reused every step)."""
+    """Device staging buffers for ``decode_step_host`` (allocated once, reused every step), carved
+    out of one block in the packed layout."""
 
     def __init__(self, desc: Desc, B: int, device):
         io = _DT_TO_TORCH[desc.io_dtype]
-        self.q = torch.empty(B, desc.H_qk or desc.H, desc.d_k, dtype=io, device=device)
-        self.k = torch.empty_like(self.q)
-        self.v = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
-        gshape = (B, desc.H, desc.d_k) if desc.op in _VEC_DECAY else (B, desc.H)
-        self.g = torch.empty(*gshape, dtype=torch.float32, device=device)
-        self.beta = torch.empty(B, desc.H, dtype=torch.float32, device=device)
+        _, total = _packed_views(desc, B, None)
+        self._block = torch.empty(total, dtype=torch.uint8, device=device)
+        v, _ = _packed_views(desc, B, self._block)
+        self.q, self.k, self.v, self.g, self.beta = v["q"], v["k"], v["v"], v["g"], v["beta"]
         self.out = torch.empty(B, desc.H, desc.d_v, dtype=io, device=device)
+        self.packed = False   # set by the caller who also passes ``packed_host_tokens`` buffers
 
     def c_struct(self) -> _Staging:
-        return _Staging(*(t.data_ptr() for t in (self.q, self.k, self.v, self.g, self.beta, self.out)))
+        return _Staging(*(t.data_ptr() for t in (self.q, self.k, self.v, self.g, self.beta, self.out)),
+                        1 if self.packed else 0)
 
     def h2d_bytes(self, desc: Desc) -> int:
         ts = [self.q, self.k, self.v, self.g] + ([self.beta] if desc.op in _DELTA_RULE else [])

@@ -77,6 +77,36 @@ TokenArgs make_token_args(const deltalog_desc *d, const void *q, const void *k, 
                      d->hints};
 }
 
+size_t round256(size_t x) { return (x + 255) / 256 * 256; }
+
+// Host and staging buffers are "packed" when q, k, v, g (if the operator has a gate) and beta (delta
+// rule) follow one another in this order, each starting on the next 256-byte boundary after the
+// previous one ends, on BOTH sides: the five copies then collapse into one over the whole block.
+// Returns the block's size, or 0 when the layout is not packed.
+size_t packed_block_bytes(const deltalog_desc *d, const deltalog_staging *stg, const void *hq, const void *hk,
+                          const void *hv, const float *hg, const float *hbeta, size_t qk_vec, size_t vec,
+                          size_t gbytes, size_t units) {
+    if (!stg->packed) return 0;  // adjacency alone proves nothing: the block must be one allocation
+    const char *h = static_cast<const char *>(hq);
+    const char *s = static_cast<const char *>(stg->q);
+    size_t off = round256(qk_vec);
+    if (static_cast<const char *>(hk) != h + off || static_cast<const char *>(stg->k) != s + off) return 0;
+    off += round256(qk_vec);
+    if (static_cast<const char *>(hv) != h + off || static_cast<const char *>(stg->v) != s + off) return 0;
+    size_t end = off + vec;
+    off += round256(vec);
+    if (op_has_gate(d->op)) {
+        if (reinterpret_cast<const char *>(hg) != h + off || reinterpret_cast<const char *>(stg->g) != s + off) return 0;
+        end = off + gbytes;
+        off += round256(gbytes);
+    }
+    if (op_delta_rule(d->op)) {
+        if (reinterpret_cast<const char *>(hbeta) != h + off || reinterpret_cast<const char *>(stg->beta) != s + off) return 0;
+        end = off + units * sizeof(float);
+    }
+    return end;
+}
+
 StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
     StateArgs a;
     a.S_base = s->S_base;
@@ -434,14 +464,20 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
     const size_t qk_vec = (size_t)B * qk_heads(desc) * desc->d_k * esz;
     const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
     if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
-    bool ok = cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (op_has_gate(desc->op))
-        ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-    if (op_delta_rule(desc->op))
-        ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s) ==
-                       cudaSuccess;
+    bool ok = true;
+    if (const size_t block = packed_block_bytes(desc, staging, host_q, host_k, host_v, host_g, host_beta, qk_vec, vec,
+                                                gbytes, units)) {
+        ok = cudaMemcpyAsync(staging->q, host_q, block, cudaMemcpyHostToDevice, s) == cudaSuccess;  // one copy
+    } else {
+        ok = cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        if (op_has_gate(desc->op))
+            ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+        if (op_delta_rule(desc->op))
+            ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s) ==
+                           cudaSuccess;
+    }
     if (!ok) return DELTALOG_ERR_CUDA;
     if (int rc = deltalog_decode_step(desc, state, staging->q, staging->k, staging->v, staging->g,
                                       staging->beta, u_bonus, slot_idx, B, staging->out, stream))
@@ -477,14 +513,19 @@ int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltal
     const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
     // copy-in stream: the staging inputs are free once the kernel that last read them is done
     bool ok = cudaStreamWaitEvent(s_in, e_cmp, 0) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    if (op_has_gate(desc->op))
-        ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
-    if (op_delta_rule(desc->op))
-        ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s_in) ==
-                       cudaSuccess;
+    if (const size_t block = packed_block_bytes(desc, staging, host_q, host_k, host_v, host_g, host_beta, qk_vec, vec,
+                                                gbytes, units)) {
+        ok = ok && cudaMemcpyAsync(staging->q, host_q, block, cudaMemcpyHostToDevice, s_in) == cudaSuccess;  // one copy
+    } else {
+        ok = ok && cudaMemcpyAsync(staging->q, host_q, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(staging->k, host_k, qk_vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(staging->v, host_v, vec, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        if (op_has_gate(desc->op))
+            ok = ok && cudaMemcpyAsync(staging->g, host_g, gbytes, cudaMemcpyHostToDevice, s_in) == cudaSuccess;
+        if (op_delta_rule(desc->op))
+            ok = ok && cudaMemcpyAsync(staging->beta, host_beta, units * sizeof(float), cudaMemcpyHostToDevice, s_in) ==
+                           cudaSuccess;
+    }
     ok = ok && cudaEventRecord(e_in, s_in) == cudaSuccess;
     // compute stream: inputs landed, and the previous output of this staging set has been read back
     ok = ok && cudaStreamWaitEvent(s_cmp, e_in, 0) == cudaSuccess;

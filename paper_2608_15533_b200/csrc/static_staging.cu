@@ -65,6 +65,7 @@ extern "C" int deltalog_decode_step_host_static(const deltalog_desc *desc, const
     stg.g = reinterpret_cast<float *>(p + 2 * qk + vo);
     stg.beta = reinterpret_cast<float *>(p + 2 * qk + vo + gb);
     stg.out = p + 2 * qk + vo + gb + bb;
+    stg.packed = 0;  // nothing is known about the caller's host buffers
     // The area keeps whatever the previous call left behind.  Rows the kernel skips (padding, bad
     // slot, full log) are not written, so the output region is cleared first: those rows read back
     // as zeros instead of as the previous call's output.

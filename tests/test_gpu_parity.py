@@ -414,3 +414,35 @@ def test_chained_launches_are_bit_identical(op, d):
         assert int(state.status.item()) == 0
         results.append((torch.stack(outs), state.S_base.clone()))
     assert torch.equal(results[0][0], results[1][0]) and torch.equal(results[0][1], results[1][1])
+
+
+@pytest.mark.parametrize("op", [GDN, KDA, RWKV6])
+def test_packed_host_buffers_travel_in_one_copy_and_give_the_same_result(op):
+    """Host tokens and staging buffers laid out back to back (256-byte aligned) are copied as one
+    block; the result is that of the device entry point."""
+    import paper_2608_15533_b200 as dl
+
+    wl = small(op, 64, torch.bfloat16, batch=5, H=3, steps=3)
+    src = workloads.TokenSource(wl, device="cpu")
+    S0 = src.initial_state().to(DEV)
+    bonus = src.bonus()
+    bonus = bonus.to(DEV) if bonus is not None else None
+    desc = make_desc(wl, 4)
+    st_h, st_d = dl.State(desc, S0.clone()), dl.State(desc, S0.clone())
+    staging = dl.HostStaging(desc, wl.batch, DEV)
+    staging.packed = True
+    host = dl.packed_host_tokens(desc, wl.batch)
+    assert host["k"].data_ptr() - host["q"].data_ptr() == staging.k.data_ptr() - staging.q.data_ptr()
+    host_out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()
+    for _ in range(wl.steps):
+        tok = src.token()
+        for name in ("q", "k", "v", "g", "beta"):
+            if tok[name] is not None:
+                host[name].copy_(tok[name])
+        dl.decode_step_host(desc, st_h, staging, host["q"], host["k"], host["v"], host["g"],
+                            host["beta"] if tok["beta"] is not None else None, host_out, u_bonus=bonus)
+        ref = dl.decode_step(desc, st_d, *(tok[n].to(DEV) for n in ("q", "k", "v", "g")),
+                             beta=tok["beta"].to(DEV) if tok["beta"] is not None else None, u_bonus=bonus)
+        torch.cuda.synchronize()
+        assert torch.equal(host_out.to(DEV), ref)
+    assert torch.equal(st_h.U_log, st_d.U_log) and torch.equal(st_h.log_len, st_d.log_len)
