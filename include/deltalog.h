@@ -24,7 +24,9 @@
  *
  * General rules for every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller; descriptor structs are HOST
- *     memory, read during the call only.  The library allocates nothing and keeps no state.
+ *     memory, read during the call only.  The library allocates nothing and keeps no state about
+ *     the caller's tensors (it only remembers, per device, facts it queried and kernel attributes it
+ *     set).
  *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default stream)
  *     and never synchronise.
  *   - Tensors are dense, row-major in the index order written beside them, 16-byte aligned.

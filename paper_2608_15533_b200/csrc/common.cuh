@@ -9,7 +9,7 @@
 
 namespace deltalog {
 
-constexpr int kThreads = 256;  // every kernel in this library runs 256-thread CTAs
+constexpr int kThreads = 256;  // CTA size of the one-unit-per-CTA kernels at head size 128 (merge, fused step, eager)
 constexpr int kWarps = kThreads / 32;
 constexpr int kMaxCap = 64;
 
