@@ -139,6 +139,9 @@ class Rig:
         self.staggered = bool(wl.staggered)
         self.predicate_merge = False   # staggered batches: one predicate merge over the whole batch instead of listed rows
         self.phase = 0
+        # several layers with staggered fills: merges off the critical path, on a side stream
+        self.overlap_merges = (bool(wl.staggered) and layers > 1 and
+                               os.environ.get("DELTALOG_BENCH_OVERLAP", "1") != "0")
         if self.staggered:  # serving shape: rows address a shuffled slot pool, every row at its own log fill
             self.slot_idx = workloads.slot_permutation(wl).to(device)
             self.delay = ((cap - workloads.fill_offsets(wl, cap)) % cap).to(device)
@@ -266,6 +269,40 @@ def graph_steps(cap: int, staggered: bool = False) -> int:
     return cap * Rig.RING // math.gcd(cap, Rig.RING)
 
 
+def capture_steps_with_merges_on_a_side_stream(rig: Rig, n_steps: int, main: "torch.cuda.Stream"):
+    """Serving shape (several layers, staggered fills), called inside a graph capture on ``main``: the
+    token-less merge of a layer depends on nothing but that layer's own previous decode step, not on
+    activations, so it does not have to sit on the critical path between two layers.  The merges run
+    on a side stream -- merge(layer, step t) after decode(layer, step t-1) -- and each decode step only
+    waits for its own layer's merge: the merge CTAs share the SMs with the persistent decode CTA of
+    another layer (their shared memory and registers fit beside it)."""
+    side = torch.cuda.Stream(device=rig.device)
+    ev = lambda: torch.cuda.Event()
+    fork = ev()
+    fork.record(main)
+    side.wait_event(fork)
+    decoded = [None] * rig.layers          # event after the latest decode step of every layer
+    for t in range(n_steps):
+        merged = []
+        with torch.cuda.stream(side):
+            for layer in range(rig.layers):
+                if decoded[layer] is not None:
+                    side.wait_event(decoded[layer])
+                rig.stag_merge(layer)
+                merged.append(ev())
+                merged[-1].record(side)
+        with torch.cuda.stream(main):
+            for layer in range(rig.layers):
+                main.wait_event(merged[layer])
+                rig.decode(t, layer)
+                decoded[layer] = ev()
+                decoded[layer].record(main)
+        rig.phase = (rig.phase + 1) % rig.cap
+    join = ev()
+    join.record(side)
+    main.wait_event(join)
+
+
 def time_graph_loop(rig: Rig, steps: int):
     """Time exactly ``steps`` steps replayed from one CUDA graph that holds ``graph_steps`` steps
     (decode launches and the merge launches between them), the way a serving loop would run the
@@ -277,9 +314,12 @@ def time_graph_loop(rig: Rig, steps: int):
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
         with torch.cuda.graph(graph, stream=stream):
-            for t in range(g_len):
-                for layer in range(rig.layers):
-                    rig.step(t, layer)
+            if rig.overlap_merges:
+                capture_steps_with_merges_on_a_side_stream(rig, g_len, stream)
+            else:
+                for t in range(g_len):
+                    for layer in range(rig.layers):
+                        rig.step(t, layer)
         graph.replay()  # warm the replay path; a graph holds whole cycles, so every replay starts in the same phase
     torch.cuda.synchronize()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -642,7 +682,8 @@ def main():
         "config": {
             "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
             "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
-            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1" if stag
+            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1"
+                      + ("; the merges run on a side stream, overlapped with other layers' decode steps" if rig.overlap_merges and use_graph else "") if stag
                       else f"after every {cap}th step"),
             "launch": (f"one CUDA graph of {g_len} steps, replayed" if use_graph else "plain launches"),
             "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
