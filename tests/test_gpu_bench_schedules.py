@@ -69,3 +69,30 @@ def test_chained_graph_replays_equal_plain_launches():
 
     ref = run(False, False)
     assert same(ref, run(True, False)) and same(ref, run(True, True))
+
+
+def test_full_size_config1_in_the_timed_launch_configuration_against_the_oracle():
+    """Configuration 1 at full size, run exactly as bench.py times it (one CUDA graph per cycle, chained
+    decode launches, 256 steps): final state of sampled units against the fp64 oracle."""
+    import numpy as np
+    import oracle
+    from harness import TOL_STATE, f64, rel_err
+
+    wl, cap, steps = workloads.CONFIGS[1], 16, 256
+    rig = bench.Rig(wl, cap, DEV)
+    units = [(0, 0), (0, 31), (17, 5), (63, 12), (64, 0), (100, 30), (127, 31), (127, 0), (31, 16), (90, 7)]
+    ub = torch.tensor([u[0] for u in units], device=DEV)
+    uh = torch.tensor([u[1] for u in units], device=DEV)
+    rig.reset_logs()
+    S0 = f64(rig.states[0].S_base[ub, uh])
+    g_len = bench.graph_steps(cap)
+    bench.time_graph_loop(rig, steps - g_len)            # one warm-up replay + (steps - g_len) timed = `steps` steps
+    torch.cuda.synchronize()
+    assert all(s == 0 for s in rig.status()) and int(rig.states[0].log_len.abs().sum()) == 0
+    ring = rig.rings[0]
+    pick = lambda name: np.stack([f64(ring[t % rig.RING][name][ub, uh]).reshape(len(units), -1) for t in range(steps)])
+    ref = oracle.eager_rollout(wl.op, S0, pick("q"), pick("k"), pick("v"), pick("g"), beta=pick("beta")[..., 0])
+    err = rel_err(f64(rig.states[0].S_base[ub, uh]), ref["S"])
+    assert err <= TOL_STATE, f"state error {err:.3e}"
+    out_err = rel_err(f64(rig.out[ub, uh]), ref["out"][-1])
+    assert out_err <= 2e-2, f"output error {out_err:.3e}"
