@@ -93,7 +93,7 @@ merge_tc_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full) {
     if (len <= 0 || len > cap || (only_if_full && len < cap)) return;  // nothing to fold: no dense write
     const int ksteps = (len + 7) / 8;
 
-    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned char *ops = smem_raw;  // per step: A_hi | A_lo | U_hi | U_lo, 4 KiB each
     float *e_s = reinterpret_cast<float *>(smem_raw + (size_t)4 * kTcOperandBytes * tc_ksteps(cap));
     uint64_t *bar = reinterpret_cast<uint64_t *>(e_s + D);
