@@ -4,11 +4,11 @@
 // schedule.  One CTA stays resident per SM and walks over its share of the (batch row, head) units.
 // Five roles run concurrently and hand work to one another through mbarriers:
 //
-//   base producer  (1 warp)  bulk asynchronous copies (cp.async.bulk, completion counted on
+//   base producers (4 warps) bulk asynchronous copies (cp.async.bulk, completion counted on
 //                            mbarriers) of 16 KiB chunks of the fp32 base tile -- the only large
-//                            read -- into the base ring, the four chunks of a unit issued by four
-//                            lanes in lockstep; a chunk's stage is refilled the moment it has been
-//                            consumed, so the HBM stream never waits for a unit's epilogue;
+//                            read -- into the base ring, warp c bringing chunk c of every unit; a
+//                            chunk's stage is refilled the moment that chunk has been consumed, so
+//                            the HBM stream never waits for a unit's epilogue or for a whole tile;
 //   aux producer   (1 warp)  per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
 //                            token vectors q, k, v (and g, bonus where they are vectors) and a small
 //                            metadata record written by the producer (len, flags, scalar gate, beta)
@@ -33,7 +33,8 @@ namespace deltalog {
 
 constexpr int kChunkBytes = 16384;
 constexpr int kPipeConsumers = 256;                    // threads of the stream group and of the scalar group
-constexpr int kPipeThreads = 2 * kPipeConsumers + 64;  // + base-ring producer warp + aux-ring producer warp
+constexpr int kBaseWarps = 4;                          // base-ring producer warps: one per chunk of a tile
+constexpr int kPipeThreads = 2 * kPipeConsumers + 32 * (kBaseWarps + 1);  // + base producers + aux-ring producer warp
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 enum : int { kMetaSkip = 1, kMetaFull = 2 };
@@ -237,12 +238,18 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     constexpr int oQ = 0, oK = D, oMK = 2 * D, oMQ = 3 * D, oLB = 4 * D, oLN = 5 * D, oCK = 6 * D,
                   oCQ = 6 * D + kMaxCap, oSC = 6 * D + 2 * kMaxCap, oRED = 6 * D + 2 * kMaxCap + 4;
 
-    if (warp == 2 * kGroupWarps) {
-        // ================= base-ring producer: needs only the slot of each unit ==================
-        // The NCHUNK chunks of a unit are issued by NCHUNK lanes in lockstep (lane c handles chunk c).
+    if (warp >= 2 * kGroupWarps && warp < 2 * kGroupWarps + kBaseWarps) {
+        // ================= base-ring producers: need only the slot of each unit ===================
+        // Warp c brings chunk c of every unit, on its own: a stage is refilled the moment the stream
+        // group has released THAT chunk, not when the whole tile two units back has been consumed
+        // (a trace showed the ring running two tiles deep at tile granularity: issue -> first chunk
+        // 1.6 us, the stream group idle in between).  One lane per warp issues; a wait + arm + copy
+        // costs it ~350 ns, one chunk per unit and warp is well inside the budget.
+        static_assert(NCHUNK <= kBaseWarps, "one producer warp per chunk of a tile");
+        const int c = warp - 2 * kGroupWarps;
         bool dead = false;
-        int m = 0;  // chunks queued so far (warp-uniform)
-        for (int it0 = 0; it0 < n_items; it0 += 32) {
+        int m = 0;  // units queued so far (warp-uniform)
+        for (int it0 = 0; it0 < n_items && c < NCHUNK; it0 += 32) {
             int slot = -1;
             if (it0 + lane < n_items) {
                 const int item = first + (it0 + lane) * stride;
@@ -253,10 +260,10 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             for (int j = 0; j < cnt; ++j) {
                 const int s = __shfl_sync(0xffffffffu, slot, j);
                 if (s < 0) continue;
-                const int h = (first + (it0 + j) * stride) % H;
-                const char *src = reinterpret_cast<const char *>(st.S_base + ((size_t)s * H + h) * D * D);
-                if (lane < NCHUNK && !dead) {
-                    const int mm = m + lane;
+                if (lane == 0 && !dead) {
+                    const int h = (first + (it0 + j) * stride) % H;
+                    const char *src = reinterpret_cast<const char *>(st.S_base + ((size_t)s * H + h) * D * D);
+                    const int mm = m * NCHUNK + c;
                     const int stage = mm % NB;
                     const uint32_t phase = (uint32_t)(mm / NB) & 1u;
                     if (!bounded_wait(empty_base + 8u * stage, phase ^ 1u, abort_flag)) {
@@ -264,44 +271,51 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     } else {
                         const uint32_t fb = full_base + 8u * stage;
                         mbar_arrive_expect_tx(fb, kChunkBytes);
-                        bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * kChunkBytes), src + (size_t)lane * kChunkBytes,
+                        bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * kChunkBytes), src + (size_t)c * kChunkBytes,
                                       kChunkBytes, fb);
                     }
                 }
-                __syncwarp();
-                m += NCHUNK;
+                ++m;
             }
         }
-        if (__any_sync(0xffffffffu, dead) && lane == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
-    } else if (warp == 2 * kGroupWarps + 1) {
+        if (lane == 0 && dead && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+    } else if (warp == 2 * kGroupWarps + kBaseWarps) {
         // ================= aux-ring producer: metadata, live log entries, token vectors ==========
         RingPos pos;
         bool dead = false;
         long long issued = 0;
         const int io_vec = D * (int)sizeof(IO);
         // Lengths and log entries are written by the step before this one: when this kernel was
-        // launched ahead of the previous kernel's completion, wait for it here (a no-op otherwise).
-        // Everything the other roles do with global memory follows from what this warp loads.
-        asm volatile("griddepcontrol.wait;\n" ::: "memory");
+        // launched ahead of the previous kernel's completion, wait for it before the first length is
+        // read (a no-op otherwise) -- after the slot indices and the per-unit token scalars, which are
+        // inputs, have been requested.  Everything the other roles do with global memory follows from
+        // what this warp loads.
+        bool waited = false;
         for (int it0 = 0; it0 < n_items; it0 += 32) {
-            int slot = -1, len = 0, flags = kMetaSkip;
+            int slot = -1, len = 0, flags = kMetaSkip, item = 0;
             float gs = 0.f, bt = 0.f;
             if (it0 + lane < n_items) {
-                const int item = first + (it0 + lane) * stride;
+                item = first + (it0 + lane) * stride;
                 slot = tk.slot_idx ? tk.slot_idx[item / H] : item / H;
                 if (slot >= st.num_slots) {
                     if (st.status) atomicOr(st.status, DELTALOG_STATUS_BAD_SLOT);
                     slot = -1;
                 }
                 if (slot >= 0) {
-                    len = st.log_len[(size_t)slot * H + item % H];
-                    flags = 0;
-                    if (len >= cap || len < 0) {
-                        if (st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
-                        flags = kMetaFull;
-                    }
                     if (!kVecDecay && tk.g) gs = tk.g[item];  // no gate: plain linear attention
                     if (kDelta) bt = tk.beta[item];
+                }
+            }
+            if (!waited) {
+                asm volatile("griddepcontrol.wait;\n" ::: "memory");
+                waited = true;
+            }
+            if (slot >= 0) {
+                len = st.log_len[(size_t)slot * H + item % H];
+                flags = 0;
+                if (len >= cap || len < 0) {
+                    if (st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
+                    flags = kMetaFull;
                 }
             }
             const int cnt = min(32, n_items - it0);
