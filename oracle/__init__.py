@@ -57,7 +57,7 @@ def _load():
         lib.oracle_eager_rollout.restype = ctypes.c_int
         lib.oracle_eager_rollout.argtypes = [
             ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
-            dp, dp, dp, dp, dp, dp, dp, dp, dp, ctypes.c_int, ip, dp,
+            dp, dp, dp, dp, dp, dp, dp, dp, dp, ctypes.c_int, ip, dp, ctypes.c_int,
         ]
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
@@ -80,12 +80,14 @@ def _ptr(a):
     return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double)) if a is not None else None
 
 
-def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapshot_at=()):
+def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapshot_at=(), state_bf16=False):
     """Eager fp64 recurrence over ``T`` tokens for ``N`` independent (sequence, head) units.
 
     Shapes: ``S0 [N,d_k,d_v]``, ``q,k [T,N,d_k]``, ``v [T,N,d_v]``, ``lam [T,N,d_lambda]`` (log-decay;
     ``d_lambda`` = 1 for GDN / RetNet, ``d_k`` for KDA / RWKV6 / GLA; ignored for plain linear
     attention), ``beta [T,N]`` (GDN / KDA), ``bonus [N,d_k]`` (RWKV6).  ``snapshot_at``: ascending 1-based token counts.
+    ``state_bf16``: the state is kept in bfloat16 between tokens (rounded after every token; the
+    16-bit-state variant of Section 2.2's roofline remark) -- ``S0`` should then be representable.
 
     Returns ``dict(out [T,N,d_v], b [T,N,d_v], S [N,d_k,d_v], snapshots [n,N,d_k,d_v])``;
     ``b`` is the value-side factor of every token (what the log's U entries must hold).
@@ -124,7 +126,7 @@ def eager_rollout(op, S0, q, k, v, lam, beta=None, bonus=None, scale=1.0, snapsh
     rc = _load().oracle_eager_rollout(
         int(op), T, N, d_k, d_v, float(scale), _ptr(S), _ptr(q), _ptr(k), _ptr(v), _ptr(lam),
         _ptr(beta), _ptr(bonus), _ptr(out), _ptr(b), int(snaps.size),
-        snaps.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), _ptr(S_snap),
+        snaps.ctypes.data_as(ctypes.POINTER(ctypes.c_int)), _ptr(S_snap), int(bool(state_bf16)),
     )
     if rc != 0:
         raise ValueError(f"oracle_eager_rollout rejected op={op}")

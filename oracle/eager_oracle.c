@@ -41,6 +41,19 @@
 #include <omp.h>
 #endif
 
+/* The value a 16-bit (bfloat16) state element holds after a store of x: fp64 -> fp32 -> bfloat16, both
+ * round-to-nearest-even (the 16-bit-state variant of the roofline discussion in Section 2.2; the
+ * arithmetic of a token stays fp64, only what is kept between tokens is rounded).  Finite x only. */
+static double round_to_bf16(double x)
+{
+    float f = (float)x;
+    unsigned int u;
+    memcpy(&u, &f, sizeof u);
+    u = (u + 0x7fffu + ((u >> 16) & 1u)) & 0xffff0000u;
+    memcpy(&f, &u, sizeof u);
+    return (double)f;
+}
+
 enum { ORACLE_GDN = 0, ORACLE_KDA = 1, ORACLE_RWKV6 = 2, ORACLE_LINATTN = 3, ORACLE_RETNET = 4, ORACLE_GLA = 5 };
 
 /* One token of the gated delta rule (GDN: d_lambda == 1, KDA: d_lambda == d_k). */
@@ -126,6 +139,8 @@ static void rwkv6_token(int d_k, int d_v, double *S, const double *r, const doub
  *   b_rec    [T][N][d_v]     the value-side factor b_t of every token, or NULL
  *   snap_at  [n_snap]        ascending 1-based token counts after which S is recorded
  *   S_snap   [n_snap][N][d_k][d_v]
+ *   state_bf16               nonzero: the state is kept in bfloat16 between tokens (rounded after every
+ *                            token's update; the token's output is formed before the rounding)
  *
  * Units run in parallel (OpenMP); each keeps its state hot across its T tokens.
  * Returns 0, or -1 for an unknown operator.
@@ -133,7 +148,7 @@ static void rwkv6_token(int d_k, int d_v, double *S, const double *r, const doub
 int oracle_eager_rollout(int op, int T, int N, int d_k, int d_v, double scale, double *S,
                          const double *q, const double *k, const double *v, const double *lambda,
                          const double *beta, const double *bonus, double *out, double *b_rec,
-                         int n_snap, const int *snap_at, double *S_snap)
+                         int n_snap, const int *snap_at, double *S_snap, int state_bf16)
 {
     int d_lambda = (op == ORACLE_GDN || op == ORACLE_RETNET) ? 1 : (op == ORACLE_LINATTN ? 0 : d_k);
     int n;
@@ -156,6 +171,10 @@ int oracle_eager_rollout(int op, int T, int N, int d_k, int d_v, double scale, d
             else
                 delta_rule_token(d_k, d_v, d_lambda, scale, Sn, q + tn * d_k, k + tn * d_k,
                                  v + tn * d_v, lambda + tn * d_lambda, beta[tn], o, b);
+            if (state_bf16) {
+                size_t x;
+                for (x = 0; x < (size_t)d_k * d_v; ++x) Sn[x] = round_to_bf16(Sn[x]);
+            }
             while (next_snap < n_snap && snap_at[next_snap] == t + 1) {
                 memcpy(S_snap + ((size_t)next_snap * N + n) * d_k * d_v, Sn,
                        sizeof(double) * (size_t)d_k * d_v);

@@ -21,22 +21,35 @@ from __future__ import annotations
 import numpy as np
 
 GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
+
+
+def round_bf16(x) -> np.ndarray:
+    """The value a bfloat16 storage element holds after a store of ``x``: fp64 -> fp32 -> bfloat16,
+    both round-to-nearest-even, returned as fp64 (finite inputs).  Pass it as ``store_base`` for the
+    16-bit base state (the 16-bit-state variant of Section 2.2's roofline remark) or as ``store_u``."""
+    f = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32))
+    u = f.view(np.uint32).astype(np.uint64)
+    u = (u + 0x7FFF + ((u >> 16) & 1)) & 0xFFFF0000
+    return u.astype(np.uint32).view(np.float32).astype(np.float64).reshape(np.shape(x))
 ADDITIVE = (LINATTN, RETNET, GLA)  # b = v, readout from the updated state; LINATTN: lambda == 0
 
 
 class LogState:
     """Base + bounded log for ``N`` independent (sequence, head) units (Section 3.1)."""
 
-    def __init__(self, op: int, S0: np.ndarray, cap: int, store_u=None):
+    def __init__(self, op: int, S0: np.ndarray, cap: int, store_u=None, store_base=None):
         """``store_u``: optional function applied to a value-side factor when it is written into the
-        log (e.g. rounding to a 16-bit format), for studies of reduced-precision logs; None = exact."""
+        log (e.g. rounding to a 16-bit format), for studies of reduced-precision logs; None = exact.
+        ``store_base``: the same for every write of the dense base (the initial state, Eq. 5) -- the
+        base is then only re-rounded once per materialisation, not once per token."""
         S0 = np.asarray(S0, dtype=np.float64)
         self.store_u = store_u
+        self.store_base = store_base
         self.op = int(op)
         self.N, self.d_k, self.d_v = S0.shape
         self.cap = int(cap)
         self.d_lambda = 1 if self.op in (GDN, RETNET, LINATTN) else self.d_k
-        self.S_base = S0.copy()
+        self.S_base = S0.copy() if store_base is None else np.asarray(store_base(S0), dtype=np.float64).copy()
         self.lbar = np.zeros((self.N, self.d_lambda))
         self.K_log = np.zeros((self.N, self.cap, self.d_k))
         self.U_log = np.zeros((self.N, self.cap, self.d_v))
@@ -145,7 +158,7 @@ def decode_merge_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: 
         S_new = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L) + np.outer(a, b)
         if st.op != RWKV6:
             out[n] = scale * (S_new.T @ q[n])
-        st.S_base[n] = S_new
+        st.S_base[n] = S_new if st.store_base is None else st.store_base(S_new)
         st.lbar[n] = 0.0
         st.length[n] = 0
     return out
@@ -157,6 +170,7 @@ def merge(st: LogState, only_if_full: bool = False) -> None:
         L = int(st.length[n])
         if L == 0 or (only_if_full and L < st.cap):
             continue
-        st.S_base[n] = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L)
+        S_new = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L)
+        st.S_base[n] = S_new if st.store_base is None else st.store_base(S_new)
         st.lbar[n] = 0.0
         st.length[n] = 0

@@ -352,3 +352,105 @@ def test_paper_cycle_with_fused_merge_step_equals_eager(op, cap):
         out = logical.decode_merge_step(st2, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus, scale=0.9)
         np.testing.assert_allclose(out, ref["out"][t], atol=1e-12)
         np.testing.assert_allclose(st2.S_base, ref["snapshots"][t], atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# 16-bit (bfloat16) state: what is stored between tokens / between materialisations is rounded
+# ---------------------------------------------------------------------------------------------
+def test_bf16_rounding_is_round_to_nearest_even_and_matches_a_library_cast():
+    torch = pytest.importorskip("torch")
+    # hand-worked cases: bfloat16 keeps 8 significant bits, ulp(1.0) = 2^-7
+    cases = {
+        1.0: 1.0,
+        1.0 + 2.0 ** -8: 1.0,                       # tie -> even mantissa (…0)
+        1.0 + 3 * 2.0 ** -8: 1.0 + 2.0 ** -6,       # tie -> even mantissa (…10)
+        1.0 + 2.0 ** -8 + 2.0 ** -20: 1.0 + 2.0 ** -7,   # just above the tie
+        -(1.0 + 2.0 ** -8 + 2.0 ** -20): -(1.0 + 2.0 ** -7),
+        0.0: 0.0,
+        2.0 ** -20 * (1 + 2.0 ** -9): 2.0 ** -20,   # below half an ulp
+        # fp64 -> fp32 comes first: 1 + 2^-8 + 2^-40 is a tie once it has been rounded to fp32
+        1.0 + 2.0 ** -8 + 2.0 ** -40: 1.0,
+    }
+    for x, want in cases.items():
+        assert float(logical.round_bf16(np.array([x]))[0]) == want, x
+    x = np.concatenate([RNG.normal(0, 1, 4096), RNG.normal(0, 1e-3, 1024), RNG.normal(0, 300, 1024)])
+    got = logical.round_bf16(x)
+    want = torch.from_numpy(x).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(got, want)
+    # exact ties on a grid: every odd multiple of half an ulp
+    m = np.arange(129, 255, dtype=np.float64)
+    ties = (2 * m + 1) * 2.0 ** -8 / 2
+    want = torch.from_numpy(ties).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(logical.round_bf16(ties), want)
+    assert logical.round_bf16(np.zeros((2, 3))).shape == (2, 3)
+
+
+def test_eager_rollout_with_bf16_state_rounds_the_stored_state_after_every_token():
+    torch = pytest.importorskip("torch")
+    cast = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    # one token from a zero state, k = e_0, beta = 1, no decay: S_1[0, :] = v, so the stored row is cast(v)
+    dk, dv = 3, 64
+    v = RNG.normal(0, 1, (1, 1, dv))
+    k = np.zeros((1, 1, dk)); k[0, 0, 0] = 1.0
+    q = RNG.normal(0, 1, (1, 1, dk))
+    r = oracle.eager_rollout(GDN, np.zeros((1, dk, dv)), q, k, v, np.zeros((1, 1, 1)), beta=np.ones((1, 1)),
+                             state_bf16=True)
+    np.testing.assert_array_equal(r["S"][0, 0], cast(v[0, 0]))
+    np.testing.assert_array_equal(r["S"][0, 1:], 0.0)
+    np.testing.assert_allclose(r["out"][0, 0], q[0, 0, 0] * v[0, 0], atol=1e-15)   # output: before the rounding
+    # every operator: T tokens with rounding == T one-token rollouts, casting the state in between
+    for op in ALL_OPS:
+        T, N, dk, dv = 5, 2, 4, 3
+        S0, q, k, v, lam, beta, bonus = rand_inputs(op, T, N, dk, dv)
+        S0 = cast(S0)
+        got = roll(op, S0, q, k, v, lam, beta, bonus, scale=1.1, snapshot_at=range(1, T + 1), state_bf16=True)
+        S = S0
+        for t in range(T):
+            one = roll(op, S, q[t:t + 1], k[t:t + 1], v[t:t + 1], lam[t:t + 1], beta[t:t + 1], bonus, scale=1.1)
+            np.testing.assert_allclose(got["out"][t], one["out"][0], atol=1e-13)
+            S = cast(one["S"])
+            np.testing.assert_array_equal(got["snapshots"][t], S)
+        # and it is a different thing from the unrounded rollout
+        plain = roll(op, S0, q, k, v, lam, beta, bonus, scale=1.1)
+        assert np.max(np.abs(plain["S"] - got["S"])) > 1e-5
+
+
+@pytest.mark.parametrize("op", ALL_OPS)
+def test_log_schedule_with_bf16_base_rounds_once_per_materialisation(op):
+    """Between materialisations nothing is rounded: with a representable S0 the logical state equals the
+    exact eager recurrence; a merge (or the fused merge step) stores the rounded represented state."""
+    torch = pytest.importorskip("torch")
+    cast = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()
+    T, N, dk, dv, cap = 9, 2, 4, 3, 4
+    S0, q, k, v, lam, beta, bonus = rand_inputs(op, T, N, dk, dv)
+    st = logical.LogState(op, S0, cap, store_base=logical.round_bf16)
+    np.testing.assert_array_equal(st.S_base, cast(S0))             # the initial state is stored rounded
+    S_start, t_start = st.S_base.copy(), 0
+    for t in range(T):
+        if (st.length == cap).all():
+            if t == cap:      # first boundary: token-less merge
+                exact = roll(op, S_start, q[t_start:t], k[t_start:t], v[t_start:t], lam[t_start:t],
+                             beta[t_start:t], bonus)["S"]
+                logical.merge(st)
+                np.testing.assert_array_equal(st.S_base, cast(exact))
+                S_start, t_start = st.S_base.copy(), t
+            else:             # second boundary: the token is consumed by the merge step itself
+                exact = roll(op, S_start, q[t_start:t + 1], k[t_start:t + 1], v[t_start:t + 1],
+                             lam[t_start:t + 1], beta[t_start:t + 1], bonus)
+                out = logical.decode_merge_step(st, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus)
+                np.testing.assert_allclose(out, exact["out"][-1], atol=1e-12)   # output: unrounded state
+                np.testing.assert_array_equal(st.S_base, cast(exact["S"]))
+                S_start, t_start = st.S_base.copy(), t + 1
+                continue
+        out = logical.decode_step(st, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus)
+        exact = roll(op, S_start, q[t_start:t + 1], k[t_start:t + 1], v[t_start:t + 1], lam[t_start:t + 1],
+                     beta[t_start:t + 1], bonus)
+        np.testing.assert_allclose(out, exact["out"][-1], atol=1e-12)
+        np.testing.assert_allclose(logical.materialize(st), exact["S"], atol=1e-12)
+    # capacity 1 through the merge step alone rounds after every token: the eager 16-bit-state recurrence
+    st1 = logical.LogState(op, S0, 1, store_base=logical.round_bf16)
+    ref = roll(op, cast(S0), q, k, v, lam, beta, bonus, snapshot_at=range(1, T + 1), state_bf16=True)
+    for t in range(T):
+        out = logical.decode_merge_step(st1, q[t], k[t], v[t], lam[t], beta=beta[t], bonus=bonus)
+        np.testing.assert_allclose(out, ref["out"][t], atol=1e-12)
+        np.testing.assert_array_equal(st1.S_base, ref["snapshots"][t])
