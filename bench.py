@@ -105,10 +105,11 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def unit_shape(wl: workloads.Workload, ulog16: bool = False) -> traffic.UnitShape:
+def unit_shape(wl: workloads.Workload, ulog16: bool = False, base16: bool = False) -> traffic.UnitShape:
     io = 4 if wl.io_dtype == torch.float32 else 2
     ul = 4 if wl.op in (workloads.GDN, workloads.KDA) and not ulog16 else io  # b = v keeps the I/O dtype
-    return traffic.UnitShape(wl.op, wl.d, wl.d, io_bytes=io, klog_bytes=io, ulog_bytes=ul)
+    return traffic.UnitShape(wl.op, wl.d, wl.d, io_bytes=io, klog_bytes=io, ulog_bytes=ul,
+                             state_bytes=2 if base16 else 4)
 
 
 class Rig:
@@ -116,22 +117,24 @@ class Rig:
 
     RING = 8
 
-    def __init__(self, wl, cap, device, seed_offset=0, layers=1, ulog16=False):
+    def __init__(self, wl, cap, device, seed_offset=0, layers=1, ulog16=False, base16=False):
         import paper_2608_15533_b200 as dl
 
         self.dl, self.wl, self.cap, self.device, self.layers = dl, wl, cap, device, layers
         io = dl.F32 if wl.io_dtype == torch.float32 else dl.BF16
+        base = dl.BF16 if base16 else dl.F32   # the 16-bit dense state is a variant; the configurations name fp32
         self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
-                            ulog_dtype=io if ulog16 else None)
+                            ulog_dtype=io if ulog16 else None, base_dtype=base)
         # the same problem with the promise that the launch in front of a decode step leaves the base
         # alone (true for every decode step of a cycle but the first after a merge)
         self.desc_chained = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
-                                    ulog_dtype=io if ulog16 else None, hints=dl.HINT_BASE_UNTOUCHED)
+                                    ulog_dtype=io if ulog16 else None, hints=dl.HINT_BASE_UNTOUCHED, base_dtype=base)
         self.chain = os.environ.get("DELTALOG_BENCH_CHAIN", "1") != "0"
         self.states, self.rings, self.bonus = [], [], []
         for layer in range(layers):
             src = workloads.TokenSource(wl, device=device, seed=wl.seed + 1000 * seed_offset + layer)
-            self.states.append(dl.State(self.desc, src.initial_state()))
+            S0 = src.initial_state()
+            self.states.append(dl.State(self.desc, S0.to(torch.bfloat16) if base16 else S0))
             self.bonus.append(src.bonus())
             self.rings.append([src.token() for _ in range(self.RING)])
         self.out = torch.empty(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
@@ -614,6 +617,8 @@ def main():
     ap.add_argument("--cap", type=int, default=16, help="log capacity of the headline number")
     ap.add_argument("--no-graph", action="store_true", help="time plain launches instead of CUDA-graph replays")
     ap.add_argument("--no-extras", action="store_true", help="skip the capacity sweep, eager and CPU legs")
+    ap.add_argument("--state", default="fp32", choices=["fp32", "bf16"],
+                    help="dtype of the dense state; bf16 is the 16-bit-state variant (the configurations name fp32)")
     ap.add_argument("--only-hot-loop", action="store_true",
                     help="warm-up and timed loop only (for profiler captures)")
     args = ap.parse_args()
@@ -630,10 +635,11 @@ def main():
     cap = args.cap
     warmup = max(args.warmup, 3)
     layers = wl.layers
-    rig = Rig(wl, cap, device, seed_offset=rank, layers=layers)
+    base16 = args.state == "bf16"
+    rig = Rig(wl, cap, device, seed_offset=rank, layers=layers, base16=base16)
     stag = rig.staggered
     g_len = graph_steps(cap, stag)
-    u = unit_shape(wl)
+    u = unit_shape(wl, base16=base16)
     units = wl.units
 
     # ---- warm-up, then the timed region: exactly K steps ---------------------------------------
@@ -674,14 +680,14 @@ def main():
     # events bracket cap decode launches per mark in a uniform batch, one decode launch per mark in a staggered one
     dec_ms_avg = dec_ms / (n_merges * (1 if stag else cap)) if n_merges else float("nan")
     achieved = dec_bytes / (dec_ms_avg * 1e-3) / 1e9
-    traffic_ncu = NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
+    traffic_ncu = None if base16 else NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
             "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
-            "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": "fp32",
+            "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": args.state,
             "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1"
                       + ("; the merges run on a side stream, overlapped with other layers' decode steps" if rig.overlap_merges and use_graph else "") if stag
                       else f"after every {cap}th step"),
@@ -752,7 +758,7 @@ def main():
                 continue
             del rig
             torch.cuda.empty_cache()
-            rig = Rig(wl, c, device, seed_offset=rank)
+            rig = Rig(wl, c, device, seed_offset=rank, base16=base16)
             for t in range(max(c, 3)):
                 rig.decode(t);
                 if (t + 1) % c == 0:

@@ -153,20 +153,34 @@ def study_ablation(steps: int) -> dict:
 
 def study_precision(device, steps: int) -> dict:
     """The value-side log of the delta rule in fp32 (default; meets the 1e-4 state bar) against the
-    16-bit variant (does not: see tests/test_ulog_precision.py): what the smaller entries buy."""
+    16-bit variant (does not: see tests/test_ulog_precision.py): what the smaller entries buy.  And the
+    16-bit dense state (tests/test_gpu_bf16_base.py): half the dense bytes, for the log schedule and for
+    the eager kernel, per capacity -- with a smaller base the replay of the log weighs more, so the best
+    capacity moves down."""
     wl = workloads.CONFIGS[1]
     rows = []
-    for name, u16 in (("U log fp32 (default)", False), ("U log bf16 (reduced precision)", True)):
-        rig = bench.Rig(wl, 16, device, ulog16=u16)
+    variants = [("fp32 state, U log fp32 (default)", False, False, 16), ("fp32 state, U log bf16", True, False, 16)]
+    variants += [(f"bf16 state, U log fp32, cap {c}", False, True, c) for c in (4, 8, 16, 32)]
+    variants += [("bf16 state, U log bf16, cap 16", True, True, 16)]
+    for name, u16, b16, cap in variants:
+        rig = bench.Rig(wl, cap, device, ulog16=u16, base16=b16)
         ms = _split_cycle_ms(rig, steps)
         assert all(s == 0 for s in rig.status())
-        u = bench.unit_shape(wl, ulog16=u16)
-        cyc = traffic.cycle_bytes(u, 16)
-        rows.append({"variant": name, "entry_bytes": u.entry, "us_per_step": ms * 1e3,
-                     "bytes_per_unit_step": cyc["total"], "hbm_gbs": cyc["total"] * wl.units / (ms * 1e-3) / 1e9})
+        u = bench.unit_shape(wl, ulog16=u16, base16=b16)
+        cyc = traffic.cycle_bytes(u, cap)
+        row = {"variant": name, "cap": cap, "state_bytes": u.state, "entry_bytes": u.entry, "us_per_step": ms * 1e3,
+               "bytes_per_unit_step": cyc["total"], "hbm_gbs": cyc["total"] * wl.units / (ms * 1e-3) / 1e9,
+               "write_reduction_vs_eager": cyc["write_reduction"]}
+        if cap == 16 and not u16:
+            rig.reset_logs()
+            e_ms = bench.time_eager_loop(rig, rig.states[0].S_base, _steps_for(rig.RING, steps)) / _steps_for(rig.RING, steps)
+            row["eager_us_per_step"] = e_ms * 1e3
+            row["eager_hbm_gbs"] = (traffic.eager_read(u) + traffic.eager_write(u)) * wl.units / (e_ms * 1e-3) / 1e9
+            row["speedup_vs_eager_kernel"] = e_ms / ms
+        rows.append(row)
         del rig
         torch.cuda.empty_cache()
-    return {"study": "precision", "workload": wl.name, "cap": 16, "rows": rows}
+    return {"study": "precision", "workload": wl.name, "rows": rows}
 
 
 def study_multi_token(device, steps: int) -> dict:

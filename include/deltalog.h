@@ -87,6 +87,12 @@ typedef struct {
                            head h uses the q and k of head h / (H / H_qk) (grouped heads: several value
                            heads share one query/key head); q and k are then [B, H_qk, d_k] */
     int32_t hints;      /* DELTALOG_HINT_* bits, 0 = none */
+    int32_t base_dtype; /* deltalog_dtype of the dense state: S_base, and S of deltalog_eager_step.
+                           DELTALOG_F32 (0, the default) or DELTALOG_BF16 -- the 16-bit state of the
+                           roofline discussion (Section 2.2): half the dense bytes.  All arithmetic stays
+                           fp32; a bf16 state is rounded (to nearest even) only when the dense state is
+                           written: once per materialisation with the log schedule (Eq. 5), once per
+                           token with the eager step.  Requires io_dtype == DELTALOG_BF16. */
 } deltalog_desc;
 
 /*
@@ -104,7 +110,7 @@ enum { DELTALOG_HINT_BASE_UNTOUCHED = 1 };
 
 /* Physical state (Section 3.1).  Device pointers, caller-owned. d_lambda = 1 (GDN) or d_k. */
 typedef struct {
-    float *S_base;     /* [num_slots, H, d_k, d_v] fp32 dense base                                  */
+    void *S_base;      /* [num_slots, H, d_k, d_v] dense base, fp32 (or desc.base_dtype)            */
     void *K_log;       /* [num_slots, H, cap, d_k] key-side factors a_t                             */
     void *U_log;       /* [num_slots, H, cap, d_v] value-side factors b_t                           */
     float *decay_log;  /* [num_slots, H, cap, d_lambda] Lambda: cumulative log-decay snapshots, fp32 */
@@ -178,7 +184,7 @@ int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const
  * is NULL) to new requests.  The log of every head of a listed slot is emptied (log_len <- 0, which
  * also clears lbar); pending entries are discarded, not folded.  With S_init != NULL (device,
  * [n, H, d_k, d_v] fp32, e.g. the state a prefill produced) the base of listed slot i becomes
- * S_init[i]; with S_init == NULL the base is left as it is.  Other slots are untouched.  Slot
+ * S_init[i] (rounded to desc.base_dtype where that is 16-bit); with S_init == NULL the base is left as it is.  Other slots are untouched.  Slot
  * indices < 0 are skipped, indices >= num_slots set DELTALOG_STATUS_BAD_SLOT and are skipped.
  */
 int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state, const int32_t *slot_idx,
@@ -186,11 +192,11 @@ int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state,
 
 /*
  * The eager dense comparator (Section 2.3): the same token update applied directly to a dense
- * state S [num_slots, H, d_k, d_v] fp32, which is read and rewritten in full on every call.
+ * state S [num_slots, H, d_k, d_v] (fp32, or desc.base_dtype), read and rewritten in full on every call.
  * Token arguments and `out` as for deltalog_decode_step; `status` (may be NULL) receives
  * DELTALOG_STATUS_BAD_SLOT bits.
  */
-int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, const void *k,
+int deltalog_eager_step(const deltalog_desc *desc, void *S, const void *q, const void *k,
                         const void *v, const float *g, const float *beta, const float *u_bonus,
                         const int32_t *slot_idx, int32_t B, void *out, int32_t *status, void *stream);
 

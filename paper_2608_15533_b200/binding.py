@@ -44,7 +44,7 @@ class DeltalogError(RuntimeError):
 class _Desc(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("op", "num_slots", "H", "d_k", "d_v", "cap", "io_dtype", "klog_dtype", "ulog_dtype")] + \
-               [("scale", ctypes.c_float), ("H_qk", ctypes.c_int32), ("hints", ctypes.c_int32)]
+               [("scale", ctypes.c_float), ("H_qk", ctypes.c_int32), ("hints", ctypes.c_int32), ("base_dtype", ctypes.c_int32)]
 
 
 class _State(ctypes.Structure):
@@ -130,6 +130,7 @@ class Desc:
     scale: float = 1.0
     H_qk: int = 0                      # query/key heads (0 = H); a divisor of H groups value heads
     hints: int = 0                     # HINT_* bits (promises by the caller, see the header)
+    base_dtype: int = F32              # dtype of the dense state; BF16 = the 16-bit state (needs io_dtype BF16)
 
     def __post_init__(self):
         if self.klog_dtype is None:
@@ -143,7 +144,8 @@ class Desc:
 
     def c_struct(self) -> _Desc:
         key = (self.op, self.num_slots, self.H, self.d_k, self.d_v, self.cap, self.io_dtype,
-               self.klog_dtype, self.ulog_dtype, float(self.scale), int(self.H_qk), int(self.hints))
+               self.klog_dtype, self.ulog_dtype, float(self.scale), int(self.H_qk), int(self.hints),
+               int(self.base_dtype))
         cached = self.__dict__.get("_c")
         if cached is None or cached[0] != key:
             cached = (key, _Desc(*key))
@@ -157,7 +159,7 @@ class State:
     def __init__(self, desc: Desc, S_base: torch.Tensor, device=None):
         device = S_base.device if device is None else device
         n, H, cap = desc.num_slots, desc.H, desc.cap
-        assert S_base.shape == (n, H, desc.d_k, desc.d_v) and S_base.dtype == torch.float32
+        assert S_base.shape == (n, H, desc.d_k, desc.d_v) and S_base.dtype == _DT_TO_TORCH[desc.base_dtype]
         self.desc = desc
         self.S_base = S_base.contiguous()
         self.K_log = torch.zeros(n, H, cap, desc.d_k, dtype=_DT_TO_TORCH[desc.klog_dtype], device=device)
@@ -254,7 +256,8 @@ def merge(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None, only
 
 def reset_slots(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None, S_init=None, stream=None) -> None:
     """``deltalog_reset_slots``: empty the logs of the listed slots (all when ``slot_idx`` is None) and,
-    with ``S_init [n,H,d_k,d_v]``, install new base states (prefill hand-off)."""
+    with ``S_init [n,H,d_k,d_v]`` fp32, install new base states (prefill hand-off)."""
+    assert S_init is None or S_init.dtype == torch.float32
     if n is None:
         n = desc.num_slots if slot_idx is None else slot_idx.numel()
     d, s = desc.c_struct(), state.c_struct()
@@ -265,7 +268,8 @@ def reset_slots(desc: Desc, state: State, slot_idx=None, n: Optional[int] = None
 
 def eager_step(desc: Desc, S: torch.Tensor, q, k, v, g, beta=None, u_bonus=None, slot_idx=None, out=None,
                status=None, stream=None) -> torch.Tensor:
-    """``deltalog_eager_step``: the dense comparator; ``S`` is rewritten in place."""
+    """``deltalog_eager_step``: the dense comparator; ``S`` (dtype ``desc.base_dtype``) is rewritten in place."""
+    assert S.dtype == _DT_TO_TORCH[desc.base_dtype]
     B = q.shape[0]
     if out is None:
         out = torch.empty(B, desc.H, desc.d_v, dtype=q.dtype, device=q.device)

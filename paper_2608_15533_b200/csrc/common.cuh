@@ -61,6 +61,40 @@ __device__ __forceinline__ void load_vec<__nv_bfloat16, 2>(const __nv_bfloat16 *
     out[0] = __uint_as_float(v << 16), out[1] = __uint_as_float(v & 0xffff0000u);
 }
 
+// Four consecutive elements of a dense state tile as one vector access.  The state is fp32, or bf16
+// (the 16-bit state of Section 2.2: half the bytes); arithmetic is fp32 either way, and a bf16 state is
+// rounded to nearest even at the store -- the only place where precision is given up.
+template <typename BT> __device__ __forceinline__ float4 base_load4(const BT *p);
+template <> __device__ __forceinline__ float4 base_load4<float>(const float *p) {
+    return *reinterpret_cast<const float4 *>(p);
+}
+template <> __device__ __forceinline__ float4 base_load4<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    const uint2 v = *reinterpret_cast<const uint2 *>(p);
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xffff0000u));
+}
+// The same through the read-only path (tiles that this kernel never writes).
+template <typename BT> __device__ __forceinline__ float4 base_ldg4(const BT *p);
+template <> __device__ __forceinline__ float4 base_ldg4<float>(const float *p) {
+    return __ldg(reinterpret_cast<const float4 *>(p));
+}
+template <> __device__ __forceinline__ float4 base_ldg4<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(p));
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xffff0000u));
+}
+template <typename BT> __device__ __forceinline__ void base_store4(BT *p, const float4 &v);
+template <> __device__ __forceinline__ void base_store4<float>(float *p, const float4 &v) {
+    *reinterpret_cast<float4 *>(p) = v;
+}
+template <> __device__ __forceinline__ void base_store4<__nv_bfloat16>(__nv_bfloat16 *p, const float4 &v) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 w;
+    w.x = *reinterpret_cast<const uint32_t *>(&lo);
+    w.y = *reinterpret_cast<const uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = w;
+}
+
 __device__ __forceinline__ float warp_sum(float x) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
@@ -176,7 +210,7 @@ struct TokenArgs {
 };
 
 struct StateArgs {
-    float *S_base;
+    void *S_base;  // fp32 or bf16 tiles (the kernels' BT template parameter)
     void *K_log, *U_log;
     float *decay_log;
     int32_t *log_len;

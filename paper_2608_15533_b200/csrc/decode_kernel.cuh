@@ -9,8 +9,8 @@
 //               b   = v;                out = y_r + (r . (bonus . k)) v
 //   append:     K[len] = k, U[len] = b, Lambda[len] = lbar', len += 1.   S_base is never written.
 //
-// The 4*d_k*d_v bytes of the base tile are the only large read; they are requested first, as
-// 16-byte loads held in registers, before anything that depends on the (small) metadata.
+// The base tile (4*d_k*d_v bytes, half of that for a bf16 base) is the only large read; it is requested
+// first, as vector loads held in registers, before anything that depends on the (small) metadata.
 #pragma once
 
 #include "common.cuh"
@@ -43,7 +43,7 @@ __host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
 #ifndef DELTALOG_SIMPLE_CTAS
 #define DELTALOG_SIMPLE_CTAS 2
 #endif
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT = float>
 __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPLE_CTAS : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
     constexpr int NT = decode_threads<D>();
     constexpr int NW = NT / 32;
@@ -65,11 +65,11 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     const int cap = st.cap;
 
     // ---- 1. request the whole base tile (independent of every other load) -------------------
-    const float4 *Sg = reinterpret_cast<const float4 *>(st.S_base + unit * D * D);
+    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * D * D;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) s[p] = __ldg(Sg + (size_t)(p * RL + rl) * C4 + c4);
+    for (int p = 0; p < NP; ++p) s[p] = base_ldg4<BT>(Sg + ((size_t)(p * RL + rl) * C4 + c4) * 4);
 
     // Programmatic dependent launch (see DELTALOG_HINT_BASE_UNTOUCHED): the kernel queued behind this
     // one may start as this one's CTAs retire; and if this kernel itself was started early, everything

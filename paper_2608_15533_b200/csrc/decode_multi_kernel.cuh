@@ -19,7 +19,7 @@
 
 namespace deltalog {
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT = float>
 __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? 2 : 8)
 decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
     constexpr int NT = decode_threads<D>();
@@ -38,11 +38,11 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
     const int cap = st.cap;
 
     // ---- the base tile: one read for all T tokens ------------------------------------------------
-    const float4 *Sg = reinterpret_cast<const float4 *>(st.S_base + unit * D * D);
+    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * D * D;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) s[p] = __ldg(Sg + (size_t)(p * RL + rl) * C4 + c4);
+    for (int p = 0; p < NP; ++p) s[p] = base_ldg4<BT>(Sg + ((size_t)(p * RL + rl) * C4 + c4) * 4);
 
     const int len0 = st.log_len[unit];
     if (len0 < 0 || len0 + T > cap) {  // no room for all T entries: the caller merges first

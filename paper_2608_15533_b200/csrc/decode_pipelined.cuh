@@ -5,14 +5,17 @@
 // Five roles run concurrently and hand work to one another through mbarriers:
 //
 //   base producers (4 warps) bulk asynchronous copies (cp.async.bulk, completion counted on
-//                            mbarriers) of 16 KiB chunks of the fp32 base tile -- the only large
-//                            read -- into the base ring, warp c bringing chunk c of every unit; a
+//                            mbarriers) of 16 KiB chunks of the base tile (fp32: four chunks, bf16:
+//                            two) -- the only large read -- into the base ring, warp c bringing
+//                            chunk c of every unit; a
 //                            chunk's stage is refilled the moment that chunk has been consumed, so
 //                            the HBM stream never waits for a unit's epilogue or for a whole tile;
-//   aux producer   (1 warp)  per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
+//   aux producers  (2 warps) per unit: the live log entries K[0:len], U[0:len], Lambda[0:len], the
 //                            token vectors q, k, v (and g, bonus where they are vectors) and a small
 //                            metadata record written by the producer (len, flags, scalar gate, beta)
-//                            into the aux ring;
+//                            into the aux ring; the warps take the units in turn (a trace showed one
+//                            thread needing 1 - 1.5 us for a unit's seven copies beside the busy
+//                            compute warps: enough for an fp32 base tile, not for a bf16 one);
 //   stream group   (8 warps) the base pass only: the two mat-vecs S_base^T (e^lbar . k) and
 //                            S_base^T (e^lbar . q) from each chunk as it lands;
 //   prep group     (4 warps) for unit i+1: cumulative decay, decayed multipliers (handed to the
@@ -32,9 +35,18 @@
 namespace deltalog {
 
 constexpr int kChunkBytes = 16384;
+// Bytes of one base-ring stage: a whole number of tile rows, at most kChunkBytes.
+template <int D, typename BT>
+__host__ __device__ constexpr int chunk_bytes() {
+    return D * D * (int)sizeof(BT) < kChunkBytes ? D * D * (int)sizeof(BT) : kChunkBytes;
+}
 constexpr int kPipeConsumers = 256;                    // threads of the stream group and of the scalar group
 constexpr int kBaseWarps = 4;                          // base-ring producer warps: one per chunk of a tile
-constexpr int kPipeThreads = 2 * kPipeConsumers + 32 * (kBaseWarps + 1);  // + base producers + aux-ring producer warp
+#ifndef DELTALOG_AUX_WARPS
+#define DELTALOG_AUX_WARPS 2
+#endif
+constexpr int kAuxWarps = DELTALOG_AUX_WARPS;          // aux-ring producer warps: they take the units in turn
+constexpr int kPipeThreads = 2 * kPipeConsumers + 32 * (kBaseWarps + kAuxWarps);  // + base and aux producers
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 enum : int { kMetaSkip = 1, kMetaFull = 2 };
@@ -61,7 +73,9 @@ struct AuxLayout {
     }
 };
 
-// Hand-over buffer between the roles, two slots (unit i and unit i+1 are in flight together).
+// Hand-over buffer between the roles: 1 << slot_shift slots (as many units are in flight between
+// the prep group and the epilogue group; two suffice while a unit's base tile takes longer to
+// arrive than the chain prep -> stream -> epilogue takes, four are used with a 16-bit base).
 // Per slot (floats): q, k, mul_k, mul_q, lbar, lbar' [6*D], ck, cq [2*64], scalars [4]: q.k and the
 // unit's flags; then the stream group's partial sums [RL][2][D].
 template <int D>
@@ -69,20 +83,21 @@ __host__ __device__ constexpr int pipe_slot_floats() {
     return 6 * D + 2 * kMaxCap + 4 + 2 * D * (kPipeConsumers / (D / 4));
 }
 template <int D>
-__host__ __device__ constexpr int pipe_scratch_bytes() {
-    return 2 * align_up(pipe_slot_floats<D>() * 4, 128);
+__host__ __device__ constexpr int pipe_scratch_bytes(int slot_shift) {
+    return (1 << slot_shift) * align_up(pipe_slot_floats<D>() * 4, 128);
 }
-constexpr int kPipeBarrierBytes = 1024;  // mbarriers (2 x 32 + 2 x 8 + 4 at most) and the abort flags
+constexpr int kPipeBarrierBytes = 1024;  // mbarriers (2 x 32 + 2 x 8 + 4 x 4 at most) and the abort flags
 
 struct PipeCfg {
     int n_base;  // stages of the base ring
     int n_aux;   // stages of the aux ring
+    int slot_shift;  // log2 of the number of hand-over slots (1 or 2)
 };
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT = float>
 __host__ inline int pipe_smem_bytes(int cap, PipeCfg cfg) {
-    return kPipeBarrierBytes + pipe_scratch_bytes<D>() + cfg.n_aux * AuxLayout<OP, D, IO, UL>(cap).bytes +
-           cfg.n_base * kChunkBytes;
+    return kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift) + cfg.n_aux * AuxLayout<OP, D, IO, UL>(cap).bytes +
+           cfg.n_base * chunk_bytes<D, BT>();
 }
 
 // ---- mbarrier / bulk-copy primitives ---------------------------------------------------------
@@ -117,8 +132,9 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 // Wait for a phase of an mbarrier, giving up after kWaitLimitNs or as soon as the CTA aborts.
-__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+// (The polling loop is kept out of line: the kernel's roles share the SM's instruction caches, and a
+// dozen inlined copies of it were a measurable part of the instruction-fetch traffic.)
+__device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     const unsigned long long t0 = global_timer_ns();
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -130,6 +146,10 @@ __device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, vola
             }
         }
     }
+}
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return bounded_wait_slow(bar, parity, abort_flag);
 }
 
 // OR-reduction of a predicate over the consumer warps (named barrier 1), also a consumer-only barrier.
@@ -169,7 +189,7 @@ struct RingPos {  // position in a ring of n stages: stage index and phase parit
     }
 };
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT = float>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
@@ -178,10 +198,11 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     constexpr int DL = kVecDecay ? D : 1;
     constexpr int C4 = D / 4;
     constexpr int RL = kPipeConsumers / C4;          // row groups of the stream group
-    constexpr int NCHUNK = D * D * 4 / kChunkBytes;  // chunks per base tile
+    constexpr int CHB = chunk_bytes<D, BT>();        // bytes per base-ring stage
+    constexpr int NCHUNK = D * D * (int)sizeof(BT) / CHB;  // chunks per base tile
     constexpr int CH_ROWS = D / NCHUNK;              // rows per chunk
     constexpr int PPC = CH_ROWS / RL;                // rows of a chunk per stream thread
-    static_assert(PPC == 4, "the base pass is written for four rows per thread and chunk");
+    static_assert(PPC % 4 == 0 && PPC * RL * NCHUNK == D, "the base pass takes a thread's rows four at a time");
     constexpr int EPL = D / 32;                      // key channels per lane in the coefficient phase
     constexpr int kGroupWarps = kPipeConsumers / 32;
     constexpr int SLOT = align_up(pipe_slot_floats<D>() * 4, 128) / 4;  // floats per hand-over slot
@@ -191,16 +212,17 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kPipeBarrierBytes - 16);
     float *scratch = reinterpret_cast<float *>(smem + kPipeBarrierBytes);
-    unsigned char *aux_ring = smem + kPipeBarrierBytes + pipe_scratch_bytes<D>();
+    unsigned char *aux_ring = smem + kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift);
     unsigned char *base_ring = aux_ring + (size_t)cfg.n_aux * lay.bytes;
 
     const int NB = cfg.n_base, NA = cfg.n_aux;
     const uint32_t full_base = smem_addr(bars), empty_base = full_base + 8u * NB;
     const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * NA;
-    const uint32_t prep_done = empty_aux + 8u * NA;   // [2] scalar group -> stream group: multipliers ready
-    const uint32_t stream_done = prep_done + 16u;     // [2] stream group -> epilogue group: partial sums ready
-    const uint32_t coef_done = stream_done + 16u;     // [2] prep group -> epilogue group: coefficients ready
-    const uint32_t slot_free = coef_done + 16u;       // [2] epilogue group -> prep group: hand-over slot reusable
+    const int SH = cfg.slot_shift, NS = 1 << SH;      // hand-over slots; unit i uses slot i % NS in phase (i / NS) & 1
+    const uint32_t prep_done = empty_aux + 8u * NA;   // [NS] scalar group -> stream group: multipliers ready
+    const uint32_t stream_done = prep_done + 8u * NS;  // [NS] stream group -> epilogue group: partial sums ready
+    const uint32_t coef_done = stream_done + 8u * NS;  // [NS] prep group -> epilogue group: coefficients ready
+    const uint32_t slot_free = coef_done + 8u * NS;    // [NS] epilogue group -> prep group: hand-over slot reusable
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) {
@@ -212,7 +234,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             mbar_init(full_aux + 8u * i, 1);
             mbar_init(empty_aux + 8u * i, kGroupWarps);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < NS; ++i) {
             mbar_init(prep_done + 8u * i, 1);
             mbar_init(stream_done + 8u * i, kGroupWarps);
             mbar_init(coef_done + 8u * i, kGroupWarps / 2);
@@ -234,7 +256,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     const int cap = st.cap, H = st.H;
 
     // hand-over slot fields
-    auto slot_ptr = [&](int i) { return scratch + (size_t)(i & 1) * SLOT; };
+    auto slot_ptr = [&](int i) { return scratch + (size_t)(i & (NS - 1)) * SLOT; };
     constexpr int oQ = 0, oK = D, oMK = 2 * D, oMQ = 3 * D, oLB = 4 * D, oLN = 5 * D, oCK = 6 * D,
                   oCQ = 6 * D + kMaxCap, oSC = 6 * D + 2 * kMaxCap, oRED = 6 * D + 2 * kMaxCap + 4;
 
@@ -262,7 +284,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                 if (s < 0) continue;
                 if (lane == 0 && !dead) {
                     const int h = (first + (it0 + j) * stride) % H;
-                    const char *src = reinterpret_cast<const char *>(st.S_base + ((size_t)s * H + h) * D * D);
+                    const char *src = static_cast<const char *>(st.S_base) + ((size_t)s * H + h) * D * D * sizeof(BT);
                     const int mm = m * NCHUNK + c;
                     const int stage = mm % NB;
                     const uint32_t phase = (uint32_t)(mm / NB) & 1u;
@@ -270,32 +292,34 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         dead = true;
                     } else {
                         const uint32_t fb = full_base + 8u * stage;
-                        mbar_arrive_expect_tx(fb, kChunkBytes);
-                        bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * kChunkBytes), src + (size_t)c * kChunkBytes,
-                                      kChunkBytes, fb);
+                        mbar_arrive_expect_tx(fb, CHB);
+                        bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * CHB), src + (size_t)c * CHB, CHB, fb);
                     }
                 }
                 ++m;
             }
         }
         if (lane == 0 && dead && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
-    } else if (warp == 2 * kGroupWarps + kBaseWarps) {
-        // ================= aux-ring producer: metadata, live log entries, token vectors ==========
-        RingPos pos;
+    } else if (warp >= 2 * kGroupWarps + kBaseWarps) {
+        // ================= aux-ring producers: metadata, live log entries, token vectors =========
+        // Warp a takes the units a, a + kAuxWarps, ... of this CTA; a unit's stage and phase follow from
+        // its index alone, so the warps need not talk to one another.
+        const int a = warp - (2 * kGroupWarps + kBaseWarps);
         bool dead = false;
-        long long issued = 0;
+        int n_done = 0;  // own units queued so far
         const int io_vec = D * (int)sizeof(IO);
         // Lengths and log entries are written by the step before this one: when this kernel was
         // launched ahead of the previous kernel's completion, wait for it before the first length is
         // read (a no-op otherwise) -- after the slot indices and the per-unit token scalars, which are
         // inputs, have been requested.  Everything the other roles do with global memory follows from
-        // what this warp loads.
+        // what these warps load.
         bool waited = false;
-        for (int it0 = 0; it0 < n_items; it0 += 32) {
+        for (int n0 = 0; a + kAuxWarps * n0 < n_items; n0 += 32) {
             int slot = -1, len = 0, flags = kMetaSkip, item = 0;
             float gs = 0.f, bt = 0.f;
-            if (it0 + lane < n_items) {
-                item = first + (it0 + lane) * stride;
+            const int my_it = a + kAuxWarps * (n0 + lane);
+            if (my_it < n_items) {
+                item = first + my_it * stride;
                 slot = tk.slot_idx ? tk.slot_idx[item / H] : item / H;
                 if (slot >= st.num_slots) {
                     if (st.status) atomicOr(st.status, DELTALOG_STATUS_BAD_SLOT);
@@ -318,7 +342,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     flags = kMetaFull;
                 }
             }
-            const int cnt = min(32, n_items - it0);
+            const int cnt = min(32, (n_items - a - kAuxWarps * n0 + kAuxWarps - 1) / kAuxWarps);
             for (int j = 0; j < cnt; ++j) {
                 const int s = __shfl_sync(0xffffffffu, slot, j);
                 const int L = __shfl_sync(0xffffffffu, len, j);
@@ -326,18 +350,21 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                 const float gsj = __shfl_sync(0xffffffffu, gs, j);
                 const float btj = __shfl_sync(0xffffffffu, bt, j);
                 if (lane != 0 || dead) continue;
-                if (!bounded_wait(empty_aux + 8u * pos.stage, pos.phase ^ 1u, abort_flag)) {
+                const int it = a + kAuxWarps * (n0 + j);
+                const int stg = it % NA;
+                const uint32_t phase = (uint32_t)(it / NA) & 1u;
+                if (!bounded_wait(empty_aux + 8u * stg, phase ^ 1u, abort_flag)) {
                     dead = true;
                     continue;
                 }
-                unsigned char *stage = aux_ring + (size_t)pos.stage * lay.bytes;
+                unsigned char *stage = aux_ring + (size_t)stg * lay.bytes;
                 *reinterpret_cast<int4 *>(stage + lay.meta) = make_int4(L, fl, __float_as_int(gsj), __float_as_int(btj));
                 *reinterpret_cast<int *>(stage + lay.meta + 16) = s;
-                const uint32_t fa = full_aux + 8u * pos.stage;
+                const uint32_t fa = full_aux + 8u * stg;
                 if (fl != 0) {
                     mbar_arrive(fa);  // nothing to copy: the compute warps only read the flags
                 } else {
-                    const int item = first + (it0 + j) * stride;
+                    const int item = first + it * stride;
                     const size_t unit = (size_t)s * H + item % H;
                     const int kb = L * D * (int)sizeof(IO), ub = L * D * (int)sizeof(UL);
                     const int lb = kVecDecay ? L * D * 4 : align_up(L, 4) * 4;
@@ -357,21 +384,15 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     bulk_copy_g2s(sa + lay.v, static_cast<const IO *>(tk.v) + (size_t)item * D, io_vec, fa);
                     if (OP == DELTALOG_RWKV6) bulk_copy_g2s(sa + lay.bonus, tk.u_bonus + (size_t)(item % H) * D, D * 4, fa);
                 }
-                pos.advance(NA);
-                ++issued;
+                ++n_done;
             }
         }
         if (lane == 0 && dead) {
+            // wait (bounded) for this warp's copies still in flight: its last own units, at most one per stage
             if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
-            const int back = (int)min((long long)NA, issued);
-            for (int i = 0; i < back; ++i) {
-                int stg = pos.stage - 1 - i;
-                uint32_t ph = pos.phase;
-                if (stg < 0) {
-                    stg += NA;
-                    ph ^= 1u;
-                }
-                bounded_wait(full_aux + 8u * stg, ph, abort_flag + 1);
+            for (int i = 0; i < n_done && kAuxWarps * i < NA; ++i) {  // units within NA of the newest: distinct stages
+                const int it = a + kAuxWarps * (n_done - 1 - i);
+                bounded_wait(full_aux + 8u * (it % NA), (uint32_t)(it / NA) & 1u, abort_flag + 1);
             }
         }
     } else if (warp < kGroupWarps) {
@@ -381,13 +402,17 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         const int c4 = tid % C4, rl = tid / C4;
         RingPos bpos;
         for (int it = 0; it < n_items; ++it) {
-            const uint32_t par = (uint32_t)(it >> 1) & 1u;
-            if (!bounded_wait(prep_done + 8u * (it & 1), par, abort_flag)) break;
+            const uint32_t par = (uint32_t)(it >> SH) & 1u;
+            if (!bounded_wait(prep_done + 8u * (it & (NS - 1)), par, abort_flag)) break;
             float *sl = slot_ptr(it);
             const int flags = __float_as_int(sl[oSC + 1]);
             if (!(flags & kMetaSkip)) {
                 const float *mk_s = sl + oMK, *mq_s = sl + oMQ;
                 float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), aq = ak;
+                // bf16 base: two rows per packed FMA (even-row and odd-row partial sums per column)
+                float2 ak2[4], aq2[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) ak2[x] = aq2[x] = make_float2(0.f, 0.f);
                 bool failed = false;
 #pragma unroll 1
                 for (int c = 0; c < NCHUNK; ++c) {
@@ -396,36 +421,73 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         break;
                     }
                     if (!(flags & kMetaFull)) {
-                        const float4 *tile =
-                            reinterpret_cast<const float4 *>(base_ring + (size_t)bpos.stage * kChunkBytes);
-                        const int r0 = c * CH_ROWS + rl * PPC;  // this thread's four consecutive rows
-                        const float4 mq4 = *reinterpret_cast<const float4 *>(mq_s + r0);
-                        float4 mk4 = mq4;
-                        if (kDelta) mk4 = *reinterpret_cast<const float4 *>(mk_s + r0);
-                        const float4 x0 = tile[(rl * PPC + 0) * C4 + c4], x1 = tile[(rl * PPC + 1) * C4 + c4];
-                        const float4 x2 = tile[(rl * PPC + 2) * C4 + c4], x3 = tile[(rl * PPC + 3) * C4 + c4];
-                        if (kDelta) {
-                            ak = fma4(mk4.x, x0, ak);
-                            ak = fma4(mk4.y, x1, ak);
-                            ak = fma4(mk4.z, x2, ak);
-                            ak = fma4(mk4.w, x3, ak);
+                        const BT *tile = reinterpret_cast<const BT *>(base_ring + (size_t)bpos.stage * CHB);
+                        if constexpr (sizeof(BT) == 2) {
+                            // With half the bytes per unit the instruction count starts to matter: rows are
+                            // taken in pairs, the pair's multipliers come from shared memory as one float2 and
+                            // one packed fp32 FMA serves both rows of a column.
+#pragma unroll
+                            for (int pg = 0; pg < PPC; pg += 2) {
+                                const int rc = rl * PPC + pg, r0 = c * CH_ROWS + rc;
+                                const float2 mq2 = *reinterpret_cast<const float2 *>(mq_s + r0);
+                                float2 mk2 = mq2;
+                                if (kDelta) mk2 = *reinterpret_cast<const float2 *>(mk_s + r0);
+                                const uint2 a = *reinterpret_cast<const uint2 *>(tile + ((rc + 0) * C4 + c4) * 4);
+                                const uint2 b = *reinterpret_cast<const uint2 *>(tile + ((rc + 1) * C4 + c4) * 4);
+                                const float2 x0 = make_float2(__uint_as_float(a.x << 16), __uint_as_float(b.x << 16));
+                                const float2 x1 = make_float2(__uint_as_float(a.x & 0xffff0000u), __uint_as_float(b.x & 0xffff0000u));
+                                const float2 x2 = make_float2(__uint_as_float(a.y << 16), __uint_as_float(b.y << 16));
+                                const float2 x3 = make_float2(__uint_as_float(a.y & 0xffff0000u), __uint_as_float(b.y & 0xffff0000u));
+                                if (kDelta) {
+                                    ak2[0] = __ffma2_rn(mk2, x0, ak2[0]);
+                                    ak2[1] = __ffma2_rn(mk2, x1, ak2[1]);
+                                    ak2[2] = __ffma2_rn(mk2, x2, ak2[2]);
+                                    ak2[3] = __ffma2_rn(mk2, x3, ak2[3]);
+                                }
+                                aq2[0] = __ffma2_rn(mq2, x0, aq2[0]);
+                                aq2[1] = __ffma2_rn(mq2, x1, aq2[1]);
+                                aq2[2] = __ffma2_rn(mq2, x2, aq2[2]);
+                                aq2[3] = __ffma2_rn(mq2, x3, aq2[3]);
+                            }
+                        } else {
+#pragma unroll
+                        for (int pg = 0; pg < PPC; pg += 4) {  // this thread's consecutive rows, four at a time
+                            const int rc = rl * PPC + pg, r0 = c * CH_ROWS + rc;
+                            const float4 mq4 = *reinterpret_cast<const float4 *>(mq_s + r0);
+                            float4 mk4 = mq4;
+                            if (kDelta) mk4 = *reinterpret_cast<const float4 *>(mk_s + r0);
+                            const float4 x0 = base_load4<BT>(tile + ((rc + 0) * C4 + c4) * 4);
+                            const float4 x1 = base_load4<BT>(tile + ((rc + 1) * C4 + c4) * 4);
+                            const float4 x2 = base_load4<BT>(tile + ((rc + 2) * C4 + c4) * 4);
+                            const float4 x3 = base_load4<BT>(tile + ((rc + 3) * C4 + c4) * 4);
+                            if (kDelta) {
+                                ak = fma4(mk4.x, x0, ak);
+                                ak = fma4(mk4.y, x1, ak);
+                                ak = fma4(mk4.z, x2, ak);
+                                ak = fma4(mk4.w, x3, ak);
+                            }
+                            aq = fma4(mq4.x, x0, aq);
+                            aq = fma4(mq4.y, x1, aq);
+                            aq = fma4(mq4.z, x2, aq);
+                            aq = fma4(mq4.w, x3, aq);
                         }
-                        aq = fma4(mq4.x, x0, aq);
-                        aq = fma4(mq4.y, x1, aq);
-                        aq = fma4(mq4.z, x2, aq);
-                        aq = fma4(mq4.w, x3, aq);
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(empty_base + 8u * bpos.stage);
                     bpos.advance(NB);
                 }
                 if (failed) break;
+                if constexpr (sizeof(BT) == 2) {
+                    ak = make_float4(ak2[0].x + ak2[0].y, ak2[1].x + ak2[1].y, ak2[2].x + ak2[2].y, ak2[3].x + ak2[3].y);
+                    aq = make_float4(aq2[0].x + aq2[0].y, aq2[1].x + aq2[1].y, aq2[2].x + aq2[2].y, aq2[3].x + aq2[3].y);
+                }
                 float4 *red4 = reinterpret_cast<float4 *>(sl + oRED);
                 if (kDelta) red4[(rl * 2 + 0) * C4 + c4] = ak;
                 red4[(rl * 2 + 1) * C4 + c4] = aq;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(stream_done + 8u * (it & 1));
+            if (lane == 0) mbar_arrive(stream_done + 8u * (it & (NS - 1)));
         }
     } else {
         // ================= scalar groups ==========================================================
@@ -442,7 +504,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             for (int j = 0; j < n_items; ++j) {
                 const int stg = j % NA;
                 bool got = bounded_wait(full_aux + 8u * stg, (uint32_t)(j / NA) & 1u, abort_flag);
-                got = got && bounded_wait(slot_free + 8u * (j & 1), ((uint32_t)(j >> 1) & 1u) ^ 1u, abort_flag);
+                got = got && bounded_wait(slot_free + 8u * (j & (NS - 1)), ((uint32_t)(j >> SH) & 1u) ^ 1u, abort_flag);
                 if (group_any(!got, 1)) {
                     alive = false;
                     break;
@@ -474,7 +536,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     }
                     if (gtid == 0) sl[oSC + 1] = __int_as_float(0);
                     group_sync(1);
-                    if (gtid == 0) mbar_arrive(prep_done + 8u * (j & 1));  // the stream group may start on this unit
+                    if (gtid == 0) mbar_arrive(prep_done + 8u * (j & (NS - 1)));  // the stream group may start on this unit
 
                     // key-side replay coefficients: each lane owns EPL consecutive key channels; a warp
                     // takes entries gwarp, gwarp+4, ... two at a time so that their reductions overlap
@@ -536,20 +598,20 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     }
                 } else if (gtid == 0) {
                     sl[oSC + 1] = __int_as_float(flags);
-                    mbar_arrive(prep_done + 8u * (j & 1));
+                    mbar_arrive(prep_done + 8u * (j & (NS - 1)));
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(coef_done + 8u * (j & 1));  // this warp's coefficients are in the slot
+                    mbar_arrive(coef_done + 8u * (j & (NS - 1)));  // this warp's coefficients are in the slot
                     mbar_arrive(empty_aux + 8u * stg);      // ... and it is done with the unit's aux stage
                 }
             }
         } else {
             for (int it = 0; it < n_items; ++it) {
                 const int stg = it % NA;
-                const uint32_t par = (uint32_t)(it >> 1) & 1u;
-                bool got = bounded_wait(stream_done + 8u * (it & 1), par, abort_flag);
-                got = got && bounded_wait(coef_done + 8u * (it & 1), par, abort_flag);
+                const uint32_t par = (uint32_t)(it >> SH) & 1u;
+                bool got = bounded_wait(stream_done + 8u * (it & (NS - 1)), par, abort_flag);
+                got = got && bounded_wait(coef_done + 8u * (it & (NS - 1)), par, abort_flag);
                 got = got && bounded_wait(full_aux + 8u * stg, (uint32_t)(it / NA) & 1u, abort_flag);
                 if (group_any(!got, 2)) {
                     alive = false;
@@ -600,7 +662,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(slot_free + 8u * (it & 1));  // the prep group may reuse the hand-over slot
+                    mbar_arrive(slot_free + 8u * (it & (NS - 1)));  // the prep group may reuse the hand-over slot
                     mbar_arrive(empty_aux + 8u * stg);       // this warp is done with the unit's aux stage
                 }
             }

@@ -45,6 +45,9 @@ int validate_desc(const deltalog_desc *d) {
                                            : d->ulog_dtype == d->io_dtype;
     if (!u_ok) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     if (d->cap < 1 || d->cap > kMaxCap) return DELTALOG_ERR_CAP_RANGE;
+    if (d->base_dtype != DELTALOG_F32 && d->base_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
+    // the 16-bit dense state is built for the 16-bit I/O configurations only
+    if (d->base_dtype == DELTALOG_BF16 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
     return DELTALOG_OK;
 }
 
@@ -198,7 +201,7 @@ int env_int(const char *name, int dflt) {
     return v ? std::atoi(v) : dflt;
 }
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT>
 int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
     static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
     static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
@@ -212,35 +215,45 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
     // Head size 64: a unit is a single 16 KiB chunk and the per-unit hand-overs of the pipeline cost
     // more than they hide, so the one-CTA-per-unit kernel is the faster one there (measured).
     bool pipelined = impl != 1 && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0) && (D == 128 || impl == 2);
-    PipeCfg cfg{0, 0};
+    constexpr int kStage = chunk_bytes<D, BT>();
+    // hand-over slots: two while the base tile's arrival sets the pace; with a 16-bit base the chain
+    // prep -> stream -> epilogue is the longer one and four units are kept in flight
+    static const int env_slots = env_int("DELTALOG_PIPE_SLOTS", 0);
+    PipeCfg cfg{0, 0, env_slots == 4 ? 2 : env_slots == 2 ? 1 : (sizeof(BT) == 2 ? 2 : 1)};
     int ctas = env_ctas > 0 ? env_ctas : 1;
     if (pipelined) {
         const int aux = AuxLayout<OP, D, IO, UL>(st.cap).bytes;
-        const int fixed = kPipeBarrierBytes + pipe_scratch_bytes<D>();
-        const int want_base = env_base > 0 ? env_base : 8;  // 128 KiB in flight per SM saturates HBM
+        const int fixed = kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift);
+        // fp32 base: 128 KiB of base tiles in flight per SM saturate HBM, four aux stages (two are held by
+        // the scalar groups, the rest is prefetch).  16-bit base: units pass twice as fast and up to four sit
+        // between the prep and the epilogue group, so more aux stages and a somewhat shorter base ring.
+        const bool b16 = sizeof(BT) == 2;
+        const int want_base = env_base > 0 ? env_base : (b16 ? 5 : 8) * (kChunkBytes / kStage);
+        const int want_aux = env_aux > 0 ? env_aux : (b16 ? 6 : 4);
         for (; ctas >= 1; --ctas) {
             int budget = dev.smem_per_sm / ctas - 1024;
             if (budget > dev.smem_optin) budget = dev.smem_optin;
             // aux stages: two are held by the scalar group (unit i and i+1), the rest is prefetch
-            for (cfg.n_aux = env_aux > 0 ? env_aux : 4; cfg.n_aux >= 2; --cfg.n_aux) {
-                cfg.n_base = (budget - fixed - cfg.n_aux * aux) / kChunkBytes;
+            for (cfg.n_aux = want_aux; cfg.n_aux >= 2; --cfg.n_aux) {
+                cfg.n_base = (budget - fixed - cfg.n_aux * aux) / kStage;
                 if (cfg.n_base >= want_base || (cfg.n_aux == 2 && cfg.n_base >= 2)) break;
             }
             if (cfg.n_aux >= 2) break;
         }
         if (ctas < 1) pipelined = false;
-        if (cfg.n_base > want_base) cfg.n_base = want_base;
+        if (cfg.n_base > 8 * (kChunkBytes / kStage)) cfg.n_base = 8 * (kChunkBytes / kStage);
+        if (env_base > 0 && cfg.n_base > env_base) cfg.n_base = env_base;
     }
     if (pipelined) {
-        auto kernel = decode_pipelined_kernel<OP, D, IO, UL>;
-        const int smem = pipe_smem_bytes<OP, D, IO, UL>(st.cap, cfg);
+        auto kernel = decode_pipelined_kernel<OP, D, IO, UL, BT>;
+        const int smem = pipe_smem_bytes<OP, D, IO, UL, BT>(st.cap, cfg);
         if (int rc = ensure_smem(kernel, smem)) return rc;
         const int grid = total < dev.sms * ctas ? total : dev.sms * ctas;
         if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, grid, kPipeThreads, smem, stream, st, tk, cfg);
         kernel<<<grid, kPipeThreads, smem, stream>>>(st, tk, cfg);
         return finish_launch();
     }
-    auto kernel = decode_append_kernel<OP, D, IO, UL>;
+    auto kernel = decode_append_kernel<OP, D, IO, UL, BT>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
     if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, total, decode_threads<D>(), smem, stream, st, tk);
@@ -248,16 +261,16 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT>
 int launch_decode_multi(const StateArgs &st, const TokenArgs &tk, int32_t T, cudaStream_t stream) {
-    auto kernel = decode_multi_kernel<OP, D, IO, UL>;
+    auto kernel = decode_multi_kernel<OP, D, IO, UL, BT>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
     kernel<<<tk.B * st.H, decode_threads<D>(), smem, stream>>>(st, tk, T);
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
     // DELTALOG_MERGE_TC = 1 (head size 128, no predicate): the contraction over the log entries runs
@@ -267,7 +280,7 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     // (measured on configuration 1: 110 / 119 / 142 / 215 us at capacity 4 / 16 / 32 / 64 against
     // 85 / 99 / 130 / 195 us for the packed-FMA kernel).
     static const int use_tc = env_int("DELTALOG_MERGE_TC", 0);
-    if constexpr (D == kTcD) {
+    if constexpr (D == kTcD && std::is_same<BT, float>::value) {
         if (use_tc && !only_if_full) {
             auto kernel = merge_tc_kernel<OP, IO, UL>;
             const size_t bytes = merge_tc_smem_bytes<OP, IO, UL>(st.cap);
@@ -281,20 +294,20 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     // call over a whole batch whose fills are staggered) most units are skipped: kMergePack candidates per CTA.
     const int pairs = n * st.H;
     if (only_if_full) {
-        auto kernel = merge_kernel<OP, D, IO, UL, kMergePack>;
+        auto kernel = merge_kernel<OP, D, IO, UL, kMergePack, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
         kernel<<<(pairs + kMergePack - 1) / kMergePack, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
     } else {
-        auto kernel = merge_kernel<OP, D, IO, UL, 1>;
+        auto kernel = merge_kernel<OP, D, IO, UL, 1, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
         kernel<<<pairs, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
     }
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    auto kernel = decode_merge_step_kernel<OP, D, IO, UL>;
+    auto kernel = decode_merge_step_kernel<OP, D, IO, UL, BT>;
     const size_t smem = fused_step_smem_bytes<D>(st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
     kernel<<<tk.B * st.H, kThreads, smem, stream>>>(st, tk);
@@ -302,8 +315,15 @@ int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t str
 }
 
 template <int OP, int D, typename IO>
-int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenArgs &tk, cudaStream_t stream) {
-    eager_step_kernel<OP, D, IO><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
+int launch_eager(void *S, const deltalog_desc *d, int32_t *status, const TokenArgs &tk, cudaStream_t stream) {
+    if constexpr (!std::is_same<IO, float>::value) {
+        if (d->base_dtype == DELTALOG_BF16) {
+            eager_step_kernel<OP, D, IO, __nv_bfloat16>
+                <<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
+            return finish_launch();
+        }
+    }
+    eager_step_kernel<OP, D, IO, float><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
     return finish_launch();
 }
 
@@ -332,15 +352,25 @@ int launch_eager(float *S, const deltalog_desc *d, int32_t *status, const TokenA
 
 // The value-side log keeps the I/O dtype where b = v (lossless).  For the delta rule it is fp32 by
 // default; a 16-bit U log (descriptor ulog_dtype == io_dtype == BF16) is the reduced-precision variant.
+// The dense base is fp32 unless the descriptor asks for the 16-bit state (16-bit I/O only).
 #define DELTALOG_WITH_UL(OP, IO, desc, FN, D, ...)                                                         \
+    do {                                                                                                  \
+        if constexpr (!std::is_same<IO, float>::value) {                                                  \
+            if ((desc)->base_dtype == DELTALOG_BF16) {                                                    \
+                DELTALOG_WITH_UL_BT(OP, IO, __nv_bfloat16, desc, FN, D, __VA_ARGS__);                     \
+            }                                                                                             \
+        }                                                                                                 \
+        DELTALOG_WITH_UL_BT(OP, IO, float, desc, FN, D, __VA_ARGS__);                                      \
+    } while (0)
+#define DELTALOG_WITH_UL_BT(OP, IO, BT, desc, FN, D, ...)                                                  \
     do {                                                                                                  \
         if constexpr (OpTraits<OP>::kDeltaRule) {                                                         \
             if constexpr (!std::is_same<IO, float>::value) {                                              \
-                if ((desc)->ulog_dtype != DELTALOG_F32) return FN<OP, D, IO, IO>(__VA_ARGS__);             \
+                if ((desc)->ulog_dtype != DELTALOG_F32) return FN<OP, D, IO, IO, BT>(__VA_ARGS__);         \
             }                                                                                             \
-            return FN<OP, D, IO, float>(__VA_ARGS__);                                                     \
+            return FN<OP, D, IO, float, BT>(__VA_ARGS__);                                                 \
         } else {                                                                                          \
-            return FN<OP, D, IO, IO>(__VA_ARGS__);                                                        \
+            return FN<OP, D, IO, IO, BT>(__VA_ARGS__);                                                    \
         }                                                                                                 \
     } while (0)
 
@@ -424,14 +454,18 @@ int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state,
     if (n == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (desc->d_k == 64)
-        reset_slots_kernel<64><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
-    else
-        reset_slots_kernel<128><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+    const bool b16 = desc->base_dtype == DELTALOG_BF16;
+    if (desc->d_k == 64) {
+        if (b16) reset_slots_kernel<64, __nv_bfloat16><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+        else reset_slots_kernel<64, float><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+    } else {
+        if (b16) reset_slots_kernel<128, __nv_bfloat16><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+        else reset_slots_kernel<128, float><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
+    }
     return finish_launch();
 }
 
-int deltalog_eager_step(const deltalog_desc *desc, float *S, const void *q, const void *k,
+int deltalog_eager_step(const deltalog_desc *desc, void *S, const void *q, const void *k,
                         const void *v, const float *g, const float *beta, const float *u_bonus,
                         const int32_t *slot_idx, int32_t B, void *out, int32_t *status, void *stream) {
     if (int rc = validate_desc(desc)) return rc;

@@ -1,5 +1,5 @@
-// Eager dense comparator: one CTA per (batch row, head) reads the whole fp32 state tile into
-// registers, applies the token (Eq. 3 with the operator's factors from Table 1) and writes the
+// Eager dense comparator: one CTA per (batch row, head) reads the whole state tile (fp32, or bf16 and
+// then rounded at every store, i.e. once per token) into registers, applies the token (Eq. 3 with the operator's factors from Table 1) and writes the
 // whole tile back -- the per-token read-modify-write whose write half the log schedule removes.
 //
 //   delta ops:  S' = D(lambda) S;  b = beta (v - S'^T k);  S = S' + k b^T;
@@ -11,9 +11,9 @@
 
 namespace deltalog {
 
-template <int OP, int D, typename IO>
+template <int OP, int D, typename IO, typename BT = float>
 __global__ void __launch_bounds__(kThreads, 2)
-eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *status, TokenArgs tk) {
+eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *status, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
@@ -26,11 +26,11 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
     if (!resolve_slot(tk.slot_idx, b, num_slots, status, tid, slot)) return;
     const size_t unit = (size_t)slot * H + h, row = (size_t)b * H + h;
 
-    float4 *Sg = reinterpret_cast<float4 *>(S + unit * D * D);
+    BT *Sg = static_cast<BT *>(S) + unit * D * D;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) s[p] = Sg[(size_t)(p * RL + rl) * C4 + c4];
+    for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(p * RL + rl) * C4 + c4) * 4);
 
     __shared__ __align__(16) float q_s[D], k_s[D], a_s[D], b_s[D];
     __shared__ __align__(16) float red_s[2 * D * RL];
@@ -102,7 +102,7 @@ eager_step_kernel(float *S, int32_t num_slots, int32_t H, float scale, int32_t *
             const float a = a_s[r];
             x = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
         }
-        Sg[(size_t)r * C4 + c4] = fma4(k_s[r], b4, x);
+        base_store4<BT>(Sg + ((size_t)r * C4 + c4) * 4, fma4(k_s[r], b4, x));
     }
 }
 

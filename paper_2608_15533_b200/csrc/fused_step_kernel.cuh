@@ -23,7 +23,7 @@ __host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
     return sizeof(float) * ((size_t)2 * cap * D + 5 * D + 2 * D * RL + 4);
 }
 
-template <int OP, int D, typename IO, typename UL>
+template <int OP, int D, typename IO, typename UL, typename BT = float>
 __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
@@ -38,11 +38,11 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     const size_t unit = (size_t)slot * st.H + h, row = (size_t)b * st.H + h;
     const int cap = st.cap;
 
-    float4 *Sg = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
+    BT *Sg = static_cast<BT *>(st.S_base) + unit * D * D;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) s[p] = Sg[(size_t)(rl * NP + p) * C4 + c4];
+    for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4);
 
     int len = st.log_len[unit];
     len = len < 0 ? 0 : (len > cap ? cap : len);
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
             const float a = w_s[r];
             x = make_float4(a * x.x, a * x.y, a * x.z, a * x.w);
         }
-        Sg[(size_t)r * C4 + c4] = fma4(k_s[r], b4, x);
+        base_store4<BT>(Sg + ((size_t)r * C4 + c4) * 4, fma4(k_s[r], b4, x));
     }
     if (tid == 0) st.log_len[unit] = 0;
 }

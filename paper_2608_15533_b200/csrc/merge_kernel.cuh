@@ -28,7 +28,7 @@ constexpr int kMergePack = DELTALOG_MERGE_PACK;  // candidates per CTA of a pred
 // PACK: (listed slot, head) pairs a CTA is responsible for: 1 when every listed unit is expected to
 // fold, kMergePack (strided over the grid) for predicate merges over a batch with staggered fills, where most
 // pairs are skipped.
-template <int OP, int D, typename IO, typename UL, int PACK>
+template <int OP, int D, typename IO, typename UL, int PACK, typename BT = float>
 __global__ void __launch_bounds__(kThreads, DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
@@ -77,11 +77,11 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     }
 
     // each thread owns rows [rl*NP, rl*NP + NP) x columns [4*c4, 4*c4 + 4)
-    float4 *Sg = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
+    BT *Sg = static_cast<BT *>(st.S_base) + unit * D * D;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
-    for (int p = 0; p < NP; ++p) s[p] = Sg[(size_t)(rl * NP + p) * C4 + c4];
+    for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4);
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][D]
@@ -123,13 +123,13 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
         [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP)[p4]; },
         [&](int i) { return U4[i * C4 + c4]; });
 #pragma unroll
-    for (int p = 0; p < NP; ++p) Sg[(size_t)(rl * NP + p) * C4 + c4] = s[p];
+    for (int p = 0; p < NP; ++p) base_store4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4, s[p]);
     if (tid == 0) st.log_len[unit] = 0;
     }
 }
 
 // Slot hand-over: empty the log of every head of the listed slots and, if given, install a new base.
-template <int D>
+template <int D, typename BT = float>
 __global__ void __launch_bounds__(kThreads) reset_slots_kernel(StateArgs st, const int32_t *slot_idx, const float *S_init) {
     const int i = blockIdx.x / st.H, h = blockIdx.x % st.H;
     int slot;
@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(kThreads) reset_slots_kernel(StateArgs st, con
     const size_t unit = (size_t)slot * st.H + h;
     if (S_init) {
         const float4 *src = reinterpret_cast<const float4 *>(S_init + ((size_t)i * st.H + h) * D * D);
-        float4 *dst = reinterpret_cast<float4 *>(st.S_base + unit * D * D);
-        for (int x = threadIdx.x; x < D * D / 4; x += kThreads) dst[x] = src[x];
+        BT *dst = static_cast<BT *>(st.S_base) + unit * D * D;
+        for (int x = threadIdx.x; x < D * D / 4; x += kThreads) base_store4<BT>(dst + 4 * x, src[x]);
     }
     if (threadIdx.x == 0) st.log_len[unit] = 0;
 }

@@ -119,7 +119,7 @@ merge_tc_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full) {
     // warp w: lane quarter q = w % 4 (rows 32q .. 32q+31), column half w / 4; per 16-row half hh and
     // 8-column block cb a thread holds rows 32q + 16hh + lane/4 (+8), columns 64 half + 8cb + 2(lane%4) + {0,1}
     const int q = warp & 3, half = warp >> 2;
-    float *Sg = st.S_base + unit * D * D;
+    float *Sg = static_cast<float *>(st.S_base) + unit * D * D;  // fp32 base only
     const int row_base = 32 * q + lane / 4, col_base = 64 * half + 2 * (lane % 4);
     float2 s[2][8][2];
 #pragma unroll
