@@ -296,14 +296,26 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                         bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * CHB), src + (size_t)c * CHB, CHB, fb);
                     }
                 }
-                ++m;
+                if (!dead) ++m;  // lane 0: units whose chunk was queued
             }
         }
-        if (lane == 0 && dead && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+        if (lane == 0 && dead) {
+            if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
+            // chunks this warp queued may still be in flight: wait (bounded) for those whose stage has not
+            // been reused since (within NB chunk indices of the newest) to land before the CTA may exit
+            for (int i = 0; i < m && NCHUNK * i < NB; ++i) {
+                const int mm = (m - 1 - i) * NCHUNK + c;
+                bounded_wait(full_base + 8u * (mm % NB), (uint32_t)(mm / NB) & 1u, abort_flag + 1);
+            }
+        }
     } else if (warp >= 2 * kGroupWarps + kBaseWarps) {
         // ================= aux-ring producers: metadata, live log entries, token vectors =========
         // Warp a takes the units a, a + kAuxWarps, ... of this CTA; a unit's stage and phase follow from
-        // its index alone, so the warps need not talk to one another.
+        // its index alone, so the warps need not talk to one another.  (The one-bit phase parity of the
+        // wait below stays unambiguous although a stage is awaited by different warps in turn: units are
+        // consumed strictly in order, and before warp a waits for unit i's stage it has queued unit
+        // i - kAuxWarps, so every unit up to i - kAuxWarps - NA -- which includes the user of this stage
+        // before the previous one -- has been consumed: the waiter is never two phases off.)
         const int a = warp - (2 * kGroupWarps + kBaseWarps);
         bool dead = false;
         int n_done = 0;  // own units queued so far
