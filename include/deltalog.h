@@ -1,7 +1,8 @@
 /*
  * deltalog.h -- C ABI of the DeltaLog recurrent-state decode library (sm_100a).
  *
- * The library keeps the recurrent state of a linear-attention layer as a dense fp32 base plus a
+ * The library keeps the recurrent state of a linear-attention layer as a dense base (fp32; bf16 as an
+ * option, see deltalog_desc.base_dtype) plus a
  * bounded log of compact per-token factors (Section 3.1 of the paper):
  *
  *     S_t = D(lbar) S_base + sum_{i < len} D(lbar - Lambda[i]) K[i] U[i]^T          (Eq. 6)

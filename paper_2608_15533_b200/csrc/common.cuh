@@ -11,6 +11,15 @@ namespace deltalog {
 
 constexpr int kThreads = 256;  // CTA size of the one-unit-per-CTA kernels at head size 128 (merge, fused step, eager)
 constexpr int kWarps = kThreads / 32;
+// CTA size of the materialisation kernels (merge, fused merge step): a thread holds D*D/NT elements of
+// the tile in registers, so more threads mean fewer registers each and more resident warps.
+#ifndef DELTALOG_MAT_THREADS
+#define DELTALOG_MAT_THREADS 256
+#endif
+template <int D>
+__host__ __device__ constexpr int mat_threads() {
+    return D >= 128 ? DELTALOG_MAT_THREADS : 256;
+}
 constexpr int kMaxCap = 64;
 
 // What the kernels need to know about an operator of Table 1.  The additive family shares kernels:
@@ -61,6 +70,9 @@ __device__ __forceinline__ void load_vec<__nv_bfloat16, 2>(const __nv_bfloat16 *
     out[0] = __uint_as_float(v << 16), out[1] = __uint_as_float(v & 0xffff0000u);
 }
 
+#ifndef DELTALOG_STREAM_BASE
+#define DELTALOG_STREAM_BASE 1
+#endif
 // Four consecutive elements of a dense state tile as one vector access.  The state is fp32, or bf16
 // (the 16-bit state of Section 2.2: half the bytes); arithmetic is fp32 either way, and a bf16 state is
 // rounded to nearest even at the store -- the only place where precision is given up.
@@ -73,13 +85,35 @@ template <> __device__ __forceinline__ float4 base_load4<__nv_bfloat16>(const __
     return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
                        __uint_as_float(v.y & 0xffff0000u));
 }
-// The same through the read-only path (tiles that this kernel never writes).
+// The same as a streaming load (evict-first in L2): a decode step reads every base tile exactly once,
+// hundreds of megabytes per launch, while the live log entries and the length words are read again by
+// the next step -- marking the tiles as the first to go keeps the small, reused data in the 126 MB L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(p));
+    return p;
+}
 template <typename BT> __device__ __forceinline__ float4 base_ldg4(const BT *p);
 template <> __device__ __forceinline__ float4 base_ldg4<float>(const float *p) {
+#if DELTALOG_STREAM_BASE
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;\n"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p), "l"(l2_policy_evict_first()));
+    return v;
+#else
     return __ldg(reinterpret_cast<const float4 *>(p));
+#endif
 }
 template <> __device__ __forceinline__ float4 base_ldg4<__nv_bfloat16>(const __nv_bfloat16 *p) {
+#if DELTALOG_STREAM_BASE
+    uint2 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v2.u32 {%0, %1}, [%2], %3;\n"
+                 : "=r"(v.x), "=r"(v.y)
+                 : "l"(p), "l"(l2_policy_evict_first()));
+#else
     const uint2 v = __ldg(reinterpret_cast<const uint2 *>(p));
+#endif
     return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
                        __uint_as_float(v.y & 0xffff0000u));
 }

@@ -125,6 +125,14 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uin
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// The same with an L2 eviction policy for the lines the copy brings in.
+__device__ __forceinline__ void bulk_copy_g2s_hint(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar,
+                                                   uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;\n" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ unsigned long long global_timer_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;\n" : "=l"(t));
@@ -271,6 +279,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         const int c = warp - 2 * kGroupWarps;
         bool dead = false;
         int m = 0;  // units queued so far (warp-uniform)
+        // every tile is read once per launch: first to be evicted from L2, so that the live log entries and
+        // the length words, which the next step reads again, stay there
+        const uint64_t stream_policy = l2_policy_evict_first();
         for (int it0 = 0; it0 < n_items && c < NCHUNK; it0 += 32) {
             int slot = -1;
             if (it0 + lane < n_items) {
@@ -293,7 +304,11 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     } else {
                         const uint32_t fb = full_base + 8u * stage;
                         mbar_arrive_expect_tx(fb, CHB);
+#if DELTALOG_STREAM_BASE
+                        bulk_copy_g2s_hint(smem_addr(base_ring + (size_t)stage * CHB), src + (size_t)c * CHB, CHB, fb, stream_policy);
+#else
                         bulk_copy_g2s(smem_addr(base_ring + (size_t)stage * CHB), src + (size_t)c * CHB, CHB, fb);
+#endif
                     }
                 }
                 if (!dead) ++m;  // lane 0: units whose chunk was queued

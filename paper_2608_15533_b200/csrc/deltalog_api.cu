@@ -296,11 +296,11 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     if (only_if_full) {
         auto kernel = merge_kernel<OP, D, IO, UL, kMergePack, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
-        kernel<<<(pairs + kMergePack - 1) / kMergePack, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
+        kernel<<<(pairs + kMergePack - 1) / kMergePack, mat_threads<D>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
     } else {
         auto kernel = merge_kernel<OP, D, IO, UL, 1, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
-        kernel<<<pairs, kThreads, smem, stream>>>(st, slot_idx, only_if_full, pairs);
+        kernel<<<pairs, mat_threads<D>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
     }
     return finish_launch();
 }
@@ -310,7 +310,7 @@ int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t str
     auto kernel = decode_merge_step_kernel<OP, D, IO, UL, BT>;
     const size_t smem = fused_step_smem_bytes<D>(st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<tk.B * st.H, kThreads, smem, stream>>>(st, tk);
+    kernel<<<tk.B * st.H, mat_threads<D>(), smem, stream>>>(st, tk);
     return finish_launch();
 }
 

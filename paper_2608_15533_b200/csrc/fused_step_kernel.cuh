@@ -18,18 +18,19 @@ namespace deltalog {
 
 template <int D>
 __host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
-    constexpr int RL = kThreads / (D / 4);
+    constexpr int RL = mat_threads<D>() / (D / 4);
     // A [cap][D], U [cap][D], e, q, k, w, b [D] each, partial sums [RL][2][D], scalars
     return sizeof(float) * ((size_t)2 * cap * D + 5 * D + 2 * D * RL + 4);
 }
 
 template <int OP, int D, typename IO, typename UL, typename BT = float>
-__global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
+__global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
-    constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL, EPL = D / 32;
+    constexpr int NT = mat_threads<D>();
+    constexpr int C4 = D / 4, RL = NT / C4, NP = D / RL, EPL = D / 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
     // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
     if (!kVecDecay) {
         const float lref = (len > 0 ? lold[0] : 0.f) + (tk.g ? gg[0] : 0.f);  // no gate: plain linear attention
-        for (int x = tid * 4; x < len * D; x += kThreads * 4) {
+        for (int x = tid * 4; x < len * D; x += NT * 4) {
             const float wi = expf(lref - Lg[x / D]);
             float kv[4], uv[4];
             load_vec<IO, 4>(Kg + x, kv);
@@ -76,7 +77,7 @@ __global__ void __launch_bounds__(kThreads, 2) decode_merge_step_kernel(StateArg
             *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
         }
     } else {
-        for (int x = tid; x < len * D; x += kThreads) {
+        for (int x = tid; x < len * D; x += NT) {
             const int i = x / D, j = x % D;
             const float lref = lold[j] + (kPost ? gg[j] : 0.f);
             A_s[x] = expf(lref - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);

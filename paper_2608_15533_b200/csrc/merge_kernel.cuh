@@ -29,11 +29,12 @@ constexpr int kMergePack = DELTALOG_MERGE_PACK;  // candidates per CTA of a pred
 // fold, kMergePack (strided over the grid) for predicate merges over a batch with staggered fills, where most
 // pairs are skipped.
 template <int OP, int D, typename IO, typename UL, int PACK, typename BT = float>
-__global__ void __launch_bounds__(kThreads, DELTALOG_MERGE_CTAS)
+__global__ void __launch_bounds__(mat_threads<D>(), DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
-    constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL;
+    constexpr int NT = mat_threads<D>();
+    constexpr int C4 = D / 4, RL = NT / C4, NP = D / RL;
 
     const int tid = threadIdx.x;
     const int cap = st.cap;
@@ -94,7 +95,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     const float *lbar = Lg + (size_t)(len - 1) * DL;
     // key-side weights A_ij = e^{lbar_j - Lambda_ij} K_ij and the value-side rows
     if (!kVecDecay) {  // one weight per entry: four elements per thread and pass
-        for (int x = tid * 4; x < len * D; x += kThreads * 4) {
+        for (int x = tid * 4; x < len * D; x += NT * 4) {
             const float wi = expf(lbar[0] - Lg[x / D]);
             float kv[4], uv[4];
             load_vec<IO, 4>(Kg + x, kv);
@@ -103,7 +104,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
             *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
         }
     } else {  // one weight per element (measured: the element-wise loop is the faster one here)
-        for (int x = tid; x < len * D; x += kThreads) {
+        for (int x = tid; x < len * D; x += NT) {
             const int i = x / D, j = x % D;
             A_s[x] = expf(lbar[j] - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);
             U_s[x] = to_f32(Ug[x]);
