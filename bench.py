@@ -40,10 +40,12 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
 # captures summarised under profiles/ (bytes per (sequence, head) unit; None = not captured).
-# Captured with `--cache-control none`, i.e. with L2 left as the previous launch left it, which is the
-# condition of the timed loop: part of the live log is then served by L2.  With ncu's default flush
-# before every launch the figures are 73 729 / 78 150 / 21 539 B (DRAM read == algorithmic read).
-NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 70745.0, (2, 16): 81604.0, (3, 16): 20934.0}
+# Captured with `--cache-control none` and only these two counters (one pass, so ncu neither flushes L2
+# nor saves and restores memory around the launch): L2 is as the previous launch left it, which is the
+# condition of the timed loop -- part of the live log and of the base tiles is then served by L2.  With
+# ncu's default flush before every launch the figures are 73 729 / 78 150 / 21 539 B (DRAM read ==
+# algorithmic read).
+NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 62109.0, (2, 16): 75622.0, (3, 16): 20068.0}
 
 
 def measured_peak_gbs():
