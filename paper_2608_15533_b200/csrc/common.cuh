@@ -93,6 +93,32 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(p));
     return p;
 }
+// L2 policy for the live log, which every later step of the cycle reads again: last to be evicted -- but
+// only for the fraction of its lines that L2 can hold.  A log that outgrows L2 is otherwise re-read
+// cyclically and an LRU-like policy keeps none of it; with fraction = capacity / footprint a stable
+// subset (chosen by the hardware from the address) stays resident and the rest streams.
+#ifndef DELTALOG_L2_KEEP
+#define DELTALOG_L2_KEEP 1
+#endif
+__device__ __forceinline__ uint64_t l2_policy_keep(float fraction) {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.L2::evict_first.b64 %0, %1;\n" : "=l"(p) : "f"(fraction));
+    return p;
+}
+__device__ __forceinline__ void st_hint(float *p, float v, uint64_t policy) {
+#if DELTALOG_L2_KEEP
+    asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;\n" ::"l"(p), "f"(v), "l"(policy) : "memory");
+#else
+    *p = v;
+#endif
+}
+__device__ __forceinline__ void st_hint(__nv_bfloat16 *p, __nv_bfloat16 v, uint64_t policy) {
+#if DELTALOG_L2_KEEP
+    asm volatile("st.global.L2::cache_hint.b16 [%0], %1, %2;\n" ::"l"(p), "h"(__bfloat16_as_ushort(v)), "l"(policy) : "memory");
+#else
+    *p = v;
+#endif
+}
 template <typename BT> __device__ __forceinline__ float4 base_ldg4(const BT *p);
 template <> __device__ __forceinline__ float4 base_ldg4<float>(const float *p) {
 #if DELTALOG_STREAM_BASE
@@ -144,6 +170,11 @@ __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr(smem_dst)), "l"(gmem_src)
                  : "memory");
 }
+__device__ __forceinline__ void cp_async16_hint(void *smem_dst, const void *gmem_src, uint64_t policy) {
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;\n" ::"r"(smem_addr(smem_dst)), "l"(gmem_src),
+                 "l"(policy)
+                 : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;\n" ::: "memory"); }
 
@@ -153,6 +184,17 @@ __device__ __forceinline__ void cta_cp_async(void *smem_dst, const void *gmem_sr
     char *d = static_cast<char *>(smem_dst);
     const char *s = static_cast<const char *>(gmem_src);
     for (int off = tid * 16; off < bytes; off += nthreads * 16) cp_async16(d + off, s + off);
+}
+
+__device__ __forceinline__ void cta_cp_async_hint(void *smem_dst, const void *gmem_src, int bytes, int tid, int nthreads,
+                                                  uint64_t policy) {
+    char *d = static_cast<char *>(smem_dst);
+    const char *s = static_cast<const char *>(gmem_src);
+#if DELTALOG_L2_KEEP
+    for (int off = tid * 16; off < bytes; off += nthreads * 16) cp_async16_hint(d + off, s + off, policy);
+#else
+    for (int off = tid * 16; off < bytes; off += nthreads * 16) cp_async16(d + off, s + off);
+#endif
 }
 
 __device__ __forceinline__ float4 fma4(float a, const float4 &x, const float4 &acc) {
@@ -251,6 +293,11 @@ struct StateArgs {
     int32_t *status;
     int32_t num_slots, H, cap;
     float scale;
+    float l2_keep_bytes;  // how much of the live log L2 is asked to hold on to (see l2_policy_keep)
+    // fraction of a unit's log lines to keep, when every unit of this launch holds about len + 1 entries
+    __device__ __forceinline__ float keep_fraction(int len, int total_units, int entry_bytes) const {
+        return fminf(1.f, l2_keep_bytes / ((float)total_units * (float)(len + 1) * (float)entry_bytes));
+    }
 };
 
 }  // namespace deltalog

@@ -102,9 +102,12 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
     const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
     const float *Lg = st.decay_log + unit * cap * DL;
-    cta_cp_async(K_s, Kg, len * D * (int)sizeof(IO), tid, NT);
-    cta_cp_async(U_s, Ug, len * D * (int)sizeof(UL), tid, NT);
-    if (kVecDecay) cta_cp_async(Lam_s, Lg, len * D * (int)sizeof(float), tid, NT);
+    constexpr int kEntryBytes = D * (int)(sizeof(IO) + sizeof(UL)) + DL * 4;
+    const int total_units = tk.B * st.H;
+    const uint64_t keep_rd = l2_policy_keep(st.keep_fraction(len, total_units, kEntryBytes));
+    cta_cp_async_hint(K_s, Kg, len * D * (int)sizeof(IO), tid, NT, keep_rd);
+    cta_cp_async_hint(U_s, Ug, len * D * (int)sizeof(UL), tid, NT, keep_rd);
+    if (kVecDecay) cta_cp_async_hint(Lam_s, Lg, len * D * (int)sizeof(float), tid, NT, keep_rd);
     cp_async_commit();
     if (!kVecDecay && tid < len) Lam_s[tid] = Lg[tid];
 
@@ -187,25 +190,27 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     }
     UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
     IO *og = static_cast<IO *>(tk.out) + row * D;
+    // the new entry is read again by the following steps: same L2 policy as the log's reads
+    const uint64_t keep_wr = l2_policy_keep(st.keep_fraction(len + 1, total_units, kEntryBytes));
     if (kDelta) {
         if (tid < D) {
             const float bval = tk.beta[row] * (to_f32(vg[c]) - y);
             b_s[c] = bval;
-            Uout[c] = from_f32<UL>(bval);
+            st_hint(Uout + c, from_f32<UL>(bval), keep_wr);
         }
         __syncthreads();
         if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
     } else if (active) {
         const IO v_raw = vg[c];
         og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], to_f32(v_raw), y));
-        Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+        st_hint(Uout + c, from_f32<UL>(to_f32(v_raw)), keep_wr);  // lossless: U log dtype equals the I/O dtype
     }
     if (tid < D) {
-        (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[tid] = k_raw;
-        if (kVecDecay) st.decay_log[(unit * cap + len) * DL + tid] = lnew;
+        st_hint(static_cast<IO *>(st.K_log) + (unit * cap + len) * D + tid, k_raw, keep_wr);
+        if (kVecDecay) st_hint(st.decay_log + (unit * cap + len) * DL + tid, lnew, keep_wr);
     }
     if (tid == 0) {
-        if (!kVecDecay) st.decay_log[unit * cap + len] = lnew;
+        if (!kVecDecay) st_hint(st.decay_log + unit * cap + len, lnew, keep_wr);
         st.log_len[unit] = len + 1;
     }
 }

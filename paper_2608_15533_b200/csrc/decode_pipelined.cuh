@@ -212,6 +212,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     constexpr int PPC = CH_ROWS / RL;                // rows of a chunk per stream thread
     static_assert(PPC % 4 == 0 && PPC * RL * NCHUNK == D, "the base pass takes a thread's rows four at a time");
     constexpr int EPL = D / 32;                      // key channels per lane in the coefficient phase
+    constexpr int kEntryBytes = D * (int)(sizeof(IO) + sizeof(UL)) + DL * 4;  // one log entry
     constexpr int kGroupWarps = kPipeConsumers / 32;
     constexpr int SLOT = align_up(pipe_slot_floats<D>() * 4, 128) / 4;  // floats per hand-over slot
 
@@ -404,9 +405,16 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     bulk_copy_g2s(sa + lay.k, static_cast<const IO *>(tk.k) + qk * D, io_vec, fa);
                     if (kVecDecay) bulk_copy_g2s(sa + lay.g, tk.g + (size_t)item * D, D * 4, fa);
                     if (L > 0) {
+#if DELTALOG_L2_KEEP
+                        const uint64_t keep = l2_policy_keep(st.keep_fraction(L, total, kEntryBytes));
+                        bulk_copy_g2s_hint(sa + lay.L, st.decay_log + unit * cap * DL, lb, fa, keep);
+                        bulk_copy_g2s_hint(sa + lay.K, static_cast<const IO *>(st.K_log) + unit * cap * D, kb, fa, keep);
+                        bulk_copy_g2s_hint(sa + lay.U, static_cast<const UL *>(st.U_log) + unit * cap * D, ub, fa, keep);
+#else
                         bulk_copy_g2s(sa + lay.L, st.decay_log + unit * cap * DL, lb, fa);
                         bulk_copy_g2s(sa + lay.K, static_cast<const IO *>(st.K_log) + unit * cap * D, kb, fa);
                         bulk_copy_g2s(sa + lay.U, static_cast<const UL *>(st.U_log) + unit * cap * D, ub, fa);
+#endif
                     }
                     bulk_copy_g2s(sa + lay.v, static_cast<const IO *>(tk.v) + (size_t)item * D, io_vec, fa);
                     if (OP == DELTALOG_RWKV6) bulk_copy_g2s(sa + lay.bonus, tk.u_bonus + (size_t)(item % H) * D, D * 4, fa);
@@ -672,18 +680,20 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     const IO v_raw = v_a[c];
                     UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
                     IO *og = static_cast<IO *>(tk.out) + (size_t)item * D;
+                    // the new entry is read again by the following steps: same L2 policy as the log's reads
+                    const uint64_t keep = l2_policy_keep(st.keep_fraction(len + 1, total, kEntryBytes));
                     if (kDelta) {
                         const float bval = __int_as_float(meta.w) * (to_f32(v_raw) - yk);
-                        Uout[c] = from_f32<UL>(bval);
+                        st_hint(Uout + c, from_f32<UL>(bval), keep);
                         og[c] = from_f32<IO>(st.scale * fmaf(sl[oSC], bval, yq));
                     } else {
-                        Uout[c] = from_f32<UL>(to_f32(v_raw));  // lossless: U log dtype equals the I/O dtype
+                        st_hint(Uout + c, from_f32<UL>(to_f32(v_raw)), keep);  // lossless: U log dtype equals the I/O dtype
                         og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(sl[oSC], to_f32(v_raw), yq));
                     }
-                    (static_cast<IO *>(st.K_log) + (unit * cap + len) * D)[c] = k_a[c];
-                    if (kVecDecay) st.decay_log[(unit * cap + len) * DL + c] = sl[oLN + c];
+                    st_hint(static_cast<IO *>(st.K_log) + (unit * cap + len) * D + c, k_a[c], keep);
+                    if (kVecDecay) st_hint(st.decay_log + (unit * cap + len) * DL + c, sl[oLN + c], keep);
                     if (c == 0) {
-                        if (!kVecDecay) st.decay_log[unit * cap + len] = sl[oLN];
+                        if (!kVecDecay) st_hint(st.decay_log + unit * cap + len, sl[oLN], keep);
                         st.log_len[unit] = len + 1;
                     }
                 }

@@ -110,6 +110,11 @@ size_t packed_block_bytes(const deltalog_desc *d, const deltalog_staging *stg, c
     return end;
 }
 
+int env_int(const char *name, int dflt) {
+    const char *v = std::getenv(name);
+    return v ? std::atoi(v) : dflt;
+}
+
 StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
     StateArgs a;
     a.S_base = s->S_base;
@@ -122,6 +127,8 @@ StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
     a.H = d->H;
     a.cap = d->cap;
     a.scale = d->scale;
+    static const int keep_mb = env_int("DELTALOG_L2_KEEP_MB", 40);
+    a.l2_keep_bytes = (float)keep_mb * 1048576.f;
     return a;
 }
 
@@ -196,10 +203,6 @@ const DeviceInfo &device_info() {
 
 // Tuning knobs (environment, read once): DELTALOG_DECODE_IMPL = 0 auto | 1 one-CTA-per-unit | 2 pipelined;
 // DELTALOG_CTAS_PER_SM, DELTALOG_BASE_STAGES, DELTALOG_AUX_STAGES override the pipelined kernel's shape.
-int env_int(const char *name, int dflt) {
-    const char *v = std::getenv(name);
-    return v ? std::atoi(v) : dflt;
-}
 
 template <int OP, int D, typename IO, typename UL, typename BT>
 int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
