@@ -45,7 +45,7 @@ FALLBACK_HBM_GBS = 6650.0
 # condition of the timed loop -- part of the live log and of the base tiles is then served by L2.  With
 # ncu's default flush before every launch the figures are 73 729 / 78 150 / 21 539 B (DRAM read ==
 # algorithmic read).
-NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 61094.0, (2, 16): 72345.0, (3, 16): 18635.0}
+NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 58505.0, (2, 16): 72364.0, (3, 16): 18637.0}
 
 
 def measured_peak_gbs():

@@ -282,7 +282,10 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         int m = 0;  // units queued so far (warp-uniform)
         // every tile is read once per launch: first to be evicted from L2, so that the live log entries and
         // the length words, which the next step reads again, stay there
-        const uint64_t stream_policy = l2_policy_evict_first();
+        // ... except for a fixed fraction of them (chosen by the hardware from the address), which is asked to
+        // stay: what L2 can hold beside the log need not be fetched from HBM again by the next step
+        const float pin_fraction = fminf(1.f, st.l2_pin_bytes / ((float)total * (float)(D * D) * (float)sizeof(BT)));
+        const uint64_t stream_policy = pin_fraction > 0.f ? l2_policy_keep(pin_fraction) : l2_policy_evict_first();
         for (int it0 = 0; it0 < n_items && c < NCHUNK; it0 += 32) {
             int slot = -1;
             if (it0 + lane < n_items) {

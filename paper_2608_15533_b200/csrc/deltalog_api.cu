@@ -129,6 +129,7 @@ StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
     a.scale = d->scale;
     static const int keep_mb = env_int("DELTALOG_L2_KEEP_MB", 40);
     a.l2_keep_bytes = (float)keep_mb * 1048576.f;
+    a.l2_pin_bytes = 0.f;  // set per launch by the pipelined decode kernel's launcher
     return a;
 }
 
@@ -205,7 +206,8 @@ const DeviceInfo &device_info() {
 // DELTALOG_CTAS_PER_SM, DELTALOG_BASE_STAGES, DELTALOG_AUX_STAGES override the pipelined kernel's shape.
 
 template <int OP, int D, typename IO, typename UL, typename BT>
-int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
+int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stream) {
+    StateArgs st = st_in;
     static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
     static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
     static const int env_base = env_int("DELTALOG_BASE_STAGES", 0);
@@ -248,6 +250,15 @@ int launch_decode(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream)
         if (env_base > 0 && cfg.n_base > env_base) cfg.n_base = env_base;
     }
     if (pipelined) {
+        // What L2 holds on to across steps is about half its size on this part (measured: a re-read set is
+        // served in full up to 40-60 MB and not at all from ~100 MB on).  The log comes first; where the
+        // full log leaves room, a fraction of the base tiles is asked to stay as well (config 1: 24 MB,
+        // 2-3 % per step; with more, log and tiles push each other out).  DELTALOG_L2_PIN_MB overrides.
+        static const int pin_mb = env_int("DELTALOG_L2_PIN_MB", -1);
+        constexpr float kMiB = 1048576.f;
+        const float entry = (float)(D * (sizeof(IO) + sizeof(UL)) + (OpTraits<OP>::kVecDecay ? D : 1) * 4);
+        const float full_log = (float)total * (float)st.cap * entry;
+        st.l2_pin_bytes = pin_mb >= 0 ? pin_mb * kMiB : fminf(24.f * kMiB, fmaxf(0.f, 64.f * kMiB - 0.75f * full_log));
         auto kernel = decode_pipelined_kernel<OP, D, IO, UL, BT>;
         const int smem = pipe_smem_bytes<OP, D, IO, UL, BT>(st.cap, cfg);
         if (int rc = ensure_smem(kernel, smem)) return rc;
