@@ -297,7 +297,8 @@ struct StateArgs {
     float l2_pin_bytes;   // how much of the dense base L2 is asked to hold on to across steps
     // fraction of a unit's log lines to keep, when every unit of this launch holds about len + 1 entries
     __device__ __forceinline__ float keep_fraction(int len, int total_units, int entry_bytes) const {
-        return fminf(1.f, l2_keep_bytes / ((float)total_units * (float)(len + 1) * (float)entry_bytes));
+        // (never zero: the policy instruction wants a fraction in (0, 1])
+        return fminf(1.f, fmaxf(1e-3f, l2_keep_bytes / ((float)total_units * (float)(len + 1) * (float)entry_bytes)));
     }
 };
 
