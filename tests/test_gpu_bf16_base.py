@@ -265,3 +265,49 @@ def test_16_bit_base_with_slots_blocks_of_tokens_and_reset(d):
     torch.cuda.synchronize()
     assert torch.equal(a.S_base[which.long()], S_new.to(torch.bfloat16))
     assert int(a.log_len[which.long()].abs().sum().item()) == 0 and int(a.log_len[7, 0].item()) == 1
+
+
+@pytest.mark.gpu
+def test_16_bit_base_at_the_full_size_of_configuration_1():
+    """Configuration 1's shape (128 x 32 heads, d = 128, cap 16) with the 16-bit base, launched the way the
+    benchmark launches it (a merge after every 16th step, decode steps behind a decode step chained);
+    a sample of units goes through the oracle that rounds at the same points."""
+    import paper_2608_15533_b200 as dl
+
+    base = workloads.CONFIGS[1]
+    cap, steps = 16, 3 * 16 + 5
+    wl = Workload("b16_full", base.op, base.batch, base.H, base.d, steps, (cap,))
+    src = workloads.TokenSource(wl, device="cuda")
+    S0 = src.initial_state().to(torch.bfloat16)
+    desc = dl.Desc(op=wl.op, num_slots=wl.batch, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=dl.BF16,
+                   base_dtype=dl.BF16)
+    desc_c = dl.Desc(op=wl.op, num_slots=wl.batch, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=dl.BF16,
+                     base_dtype=dl.BF16, hints=dl.HINT_BASE_UNTOUCHED)
+    state = dl.State(desc, S0.clone())
+    rng = np.random.default_rng(7)
+    picks = sorted({0, wl.batch * wl.H - 1, *rng.choice(wl.batch * wl.H, 14, replace=False).tolist()})
+    units = [(p // wl.H, p % wl.H) for p in picks]
+    ub = torch.tensor([u[0] for u in units], device="cuda")
+    uh = torch.tensor([u[1] for u in units], device="cuda")
+    rec = Recorded(units=units)
+    boundaries, got_states = [], []
+    for t in range(steps):
+        tok = src.token()
+        if t and t % cap == 0:
+            dl.merge(desc, state)
+            boundaries.append(t)
+            got_states.append(f64(state.S_base[ub, uh]))
+        out = dl.decode_step(desc if t % cap == 0 else desc_c, state, tok["q"], tok["k"], tok["v"], tok["g"],
+                             beta=tok["beta"])
+        rec.record_token(tok, out, wl)
+    dl.merge(desc, state)
+    boundaries.append(steps)
+    got_states.append(f64(state.S_base[ub, uh]))
+    torch.cuda.synchronize()
+    assert int(state.status.item()) == 0
+    q, k, v, g, beta = _arrays(rec, wl.op)
+    want_out, want_states, _ = schedule_oracle(wl.op, f64(S0[ub, uh]), q, k, v, g, beta, None, boundaries)
+    assert rel_err(np.stack(rec.out), want_out) <= TOL_OUT
+    assert_same_rounding(got_states[0], want_states[0])
+    for got, want in zip(got_states, want_states):
+        assert rel_err(got, want) <= TOL_STATE_BF16
