@@ -4,18 +4,30 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..4] [--cap C] [--impl ours|reference]
 
 One "step" is one decode token for the whole batch of the workload: the decode+append kernel, and
-the merge kernel whenever the logs are full (every ``cap`` steps), i.e. the complete hot path.
+the merge kernel whenever the logs are full (after every ``cap``-th step), i.e. the complete hot path.
+The timed region is EXACTLY K steps starting from empty logs, so it contains ``K // cap`` merges; any
+K >= 1 works.  A short region is repeated (the logs are emptied before every repetition, outside the
+timed region) and the median over the repetitions is reported; ``steps`` stays K.
 Rank 0 prints ONE JSON line.  ``value`` is (sequence*head) state updates per second with all inputs
-resident in HBM; ``e2e`` is the same metric through ``deltalog_decode_step_host`` with the token
-tensors in pinned host memory and the output read back to the host every step.
+resident in HBM; ``e2e`` is the same metric through ``deltalog_decode_step_host_overlapped`` with the
+token tensors in pinned host memory and the output read back to the host every step.
+
+``roofline`` describes the decode kernel.  Two byte counts appear side by side: ``traffic`` is DRAM
+traffic per launch measured by ncu (``profiles/dram_traffic.json``, valid only for the library build
+it was captured on -- ``null`` otherwise), and ``algorithmic_bytes_per_launch`` is what the method
+must move; since the kernels ask L2 to keep the live log, part of the algorithmic bytes never reach
+DRAM.  ``achieved`` / ``frac`` are the DRAM figures when a matching capture exists
+(``achieved_kind`` says which); the algorithmic ones are always given as ``*_algorithmic_incl_l2``.
 
 With N > 1 (one process per GPU, launched by ``torch.distributed.run``) every rank decodes its own
-shard of batch rows -- the path has no exchange step -- and the time is the maximum over ranks.
+shard of the global batch rows -- the path has no exchange step -- and the time is the maximum over
+ranks.
 """
 from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -31,21 +43,14 @@ if str(ROOT) not in sys.path:
 import torch  # noqa: E402
 
 import workloads  # noqa: E402
-from paper_2608_15533_b200 import launch, traffic  # noqa: E402
+from paper_2608_15533_b200 import launch, ncu_traffic, traffic  # noqa: E402
 
 METRIC = "state-update (seq*head)-steps/s"
 UNIT = "(seq*head)-steps/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel, from the ncu
-# captures summarised under profiles/ (bytes per (sequence, head) unit; None = not captured).
-# Captured with `--cache-control none` and only these two counters (one pass, so ncu neither flushes L2
-# nor saves and restores memory around the launch): L2 is as the previous launch left it, which is the
-# condition of the timed loop -- part of the live log and of the base tiles is then served by L2.  With
-# ncu's default flush before every launch the figures are 73 729 / 78 150 / 21 539 B (DRAM read ==
-# algorithmic read).
-NCU_DECODE_TRAFFIC_PER_UNIT = {(1, 16): 58505.0, (2, 16): 72364.0, (3, 16): 18637.0}
+TARGET_TIMED_MS = 300.0     # a short K-step region is repeated until about this much has been timed
+MAX_REPEATS, MIN_REPEATS = 25, 3
 
 
 def measured_peak_gbs():
@@ -59,55 +64,98 @@ def measured_peak_gbs():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed regions run: NVML from a thread every
+    2 ms (a K-step region can be shorter than a millisecond, far below what ``nvidia-smi -lms`` resolves),
+    ``nvidia-smi`` as the fallback.  Samples taken while ``busy`` is set count as "under load"."""
 
+    REASONS = (("hw_slowdown", 0x8), ("hw_thermal_slowdown", 0x40), ("sw_thermal_slowdown", 0x20),
+               ("sw_power_cap", 0x4))
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
-        self.rows, self.proc, self.gpu = [], None, gpu_index
+        self.gpu, self.rows, self.busy, self.stop = gpu_index, [], False, False
+        self.proc = self.thread = self.nvml = self.handle = None
+        self.sm_max = None
+
+    def _nvml_handle(self):
+        import pynvml
+
+        pynvml.nvmlInit()
+        self.nvml = pynvml
+        props = torch.cuda.get_device_properties(self.gpu)
+        uuid = getattr(props, "uuid", None)
+        if uuid is not None:
+            try:
+                return pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + str(uuid)).encode())
+            except Exception:
+                pass
+        return pynvml.nvmlDeviceGetHandleByIndex(self.gpu)
 
     def __enter__(self):
         try:
+            self.handle = self._nvml_handle()
+            self.sm_max = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.thread = threading.Thread(target=self._poll_nvml, daemon=True)
+            self.thread.start()
+            return self
+        except Exception:
+            self.handle = None
+        try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread = threading.Thread(target=self._read_smi, daemon=True)
             self.thread.start()
         except OSError:
             self.proc = None
         return self
 
-    def _read(self):
+    def _poll_nvml(self):
+        n = self.nvml
+        reasons_fn = getattr(n, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            getattr(n, "nvmlDeviceGetCurrentClocksThrottleReasons")
+        while not self.stop:
+            try:
+                sm = float(n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM))
+                mask = int(reasons_fn(self.handle))
+                self.rows.append((sm, self.sm_max, [name for name, bit in self.REASONS if mask & bit], self.busy))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def _read_smi(self):
+        names = [name for name, _ in self.REASONS]
         for line in self.proc.stdout:
-            self.rows.append([c.strip() for c in line.split(",")])
+            r = [c.strip() for c in line.split(",")]
+            try:
+                self.rows.append((float(r[0]), float(r[1]),
+                                  [nm for nm, flag in zip(names, r[3:7]) if flag.lower().startswith("active")],
+                                  self.busy))
+            except (ValueError, IndexError):
+                continue
 
     def __exit__(self, *exc):
+        self.stop = True
         if self.proc is not None:
-            time.sleep(0.15)
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=5)
             except subprocess.TimeoutExpired:
                 self.proc.kill()
+        if self.thread is not None:
             self.thread.join(timeout=2)
 
     def summary(self):
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1]))
-            except (ValueError, IndexError):
-                continue
-            for name, flag in zip(names, r[3:7]):
-                if flag.lower().startswith("active"):
-                    reasons.add(name)
-        if not sm:
+        rows = list(self.rows)
+        loaded = [r for r in rows if r[3]]
+        use = loaded if len(loaded) >= 3 else rows
+        if not use:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                "samples": len(sm)}
+        return {"sm_mhz": statistics.median(r[0] for r in use), "sm_max_mhz": max(r[1] for r in use),
+                "reasons": sorted({name for r in use for name in r[2]}), "samples": len(use),
+                "samples_under_load": len(loaded), "source": "nvml" if self.handle is not None else "nvidia-smi"}
 
 
 def unit_shape(wl: workloads.Workload, ulog16: bool = False, base16: bool = False) -> traffic.UnitShape:
@@ -130,10 +178,11 @@ class Rig:
         base = dl.BF16 if base16 else dl.F32   # the 16-bit dense state is a variant; the configurations name fp32
         self.desc = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
                             ulog_dtype=io if ulog16 else None, base_dtype=base)
-        # the same problem with the promise that the launch in front of a decode step leaves the base
-        # alone (true for every decode step of a cycle but the first after a merge)
+        # the same problem with the promise that the launch in front of a decode step writes neither the
+        # base nor the slot list (true for every decode step of a cycle but the first after a merge)
         self.desc_chained = dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io,
-                                    ulog_dtype=io if ulog16 else None, hints=dl.HINT_BASE_UNTOUCHED, base_dtype=base)
+                                    ulog_dtype=io if ulog16 else None,
+                                    hints=dl.HINT_BASE_UNTOUCHED | dl.HINT_SLOTS_STABLE, base_dtype=base)
         self.chain = os.environ.get("DELTALOG_BENCH_CHAIN", "1") != "0"
         self.states, self.rings, self.bonus = [], [], []
         for layer in range(layers):
@@ -190,9 +239,9 @@ class Rig:
             self.phase = (self.phase + 1) % self.cap
 
     def step(self, t, layer=0):
-        """One step of the hot path for one layer.  Uniform batch: decode, and the merge after every
-        cap-th step.  Staggered batch: a merge of the rows whose log is full (about 1/cap of the rows per
-        step), then decode."""
+        """Step ``t`` (counted from the last ``reset_logs``) of the hot path for one layer.  Uniform batch:
+        decode, and the merge after every cap-th step.  Staggered batch: a merge of the rows whose log is
+        full (about 1/cap of the rows per step), then decode."""
         if self.staggered:
             self.stag_merge(layer)
             self.decode(t, layer)
@@ -203,9 +252,9 @@ class Rig:
                 self.merge(layer)
 
     def reset_logs(self):
-        """Fold everything; a staggered batch is then rolled forward so that row b holds
-        (cap - delay_b) entries: rows sit out (slot -1) until their start step, real decode steps
-        fill the logs (nothing is fabricated)."""
+        """Fold everything, so that the next step is step 0 of a cycle; a staggered batch is then rolled
+        forward so that row b holds (cap - delay_b) entries: rows sit out (slot -1) until their start step,
+        real decode steps fill the logs (nothing is fabricated)."""
         for layer in range(self.layers):
             self.merge(layer, only_if_full=False)
         if self.staggered:
@@ -218,63 +267,26 @@ class Rig:
     def status(self):
         return [int(s.status.item()) for s in self.states]
 
-
-def time_cycle_loop(rig: Rig, steps: int, per_kernel: bool = True):
-    """Time exactly ``steps`` steps (decode every step, merge after every cap-th) as plain launches
-    on the current stream.  With ``per_kernel`` two events per cycle split the time into decode
-    launches and the merge launch (an event between every pair of launches would itself cost
-    several microseconds per step); returns total ms, summed decode ms, summed merge ms, merges."""
-    cap = rig.cap
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-    start, end = ev(), ev()
-    marks = []  # (event before the first decode of a cycle, event after its last decode, event after its merge)
-    launch.barrier()
-    torch.cuda.synchronize()
-    start.record()
-    for t in range(steps):
-        for layer in range(rig.layers):
-            if rig.staggered:
-                if per_kernel and layer == 0:  # one layer in `layers` carries the events
-                    marks.append([ev(), ev(), ev()])
-                    marks[-1][1].record()       # merge first here: [1] -> merge -> [2]=[0] -> decode -> end
-                    rig.stag_merge(layer)
-                    marks[-1][0].record()
-                    rig.decode(t, layer)
-                    marks[-1][2].record()
-                    rig.end_layer(layer)
-                else:
-                    rig.step(t, layer)
-                continue
-            if per_kernel and layer == 0 and t % cap == 0:
-                marks.append([ev(), None, None])
-                marks[-1][0].record()
-            rig.decode(t, layer, chained=(rig.layers == 1 and t % cap != 0))
-            if (t + 1) % cap == 0:
-                if per_kernel and layer == 0:
-                    marks[-1][1] = ev(); marks[-1][1].record()
-                rig.merge(layer)
-                if per_kernel and layer == 0:
-                    marks[-1][2] = ev(); marks[-1][2].record()
-    end.record()
-    torch.cuda.synchronize()
-    launch.barrier()
-    total = start.elapsed_time(end)
-    full = [m for m in marks if m[2] is not None]
-    if rig.staggered:  # per step: [1] merge [0] decode [2]
-        dec = sum(a.elapsed_time(c) for a, _, c in full) if per_kernel else None
-        mrg = sum(b.elapsed_time(a) for a, b, _ in full) if per_kernel else None
-    else:              # per cycle: [0] cap decodes [1] merge [2]
-        dec = sum(a.elapsed_time(b) for a, b, _ in full) if per_kernel else None
-        mrg = sum(b.elapsed_time(c) for _, b, c in full) if per_kernel else None
-    return total, dec, mrg, len(full)
+    def check_status(self, where):
+        st = self.status()
+        if any(st):
+            raise RuntimeError(f"{where}: device status bits set: {st} (1 = log full, 2 = bad slot, 4 = wait timed out)")
 
 
-def graph_steps(cap: int, staggered: bool = False) -> int:
+def merges_in(steps: int, cap: int) -> int:
+    """Merges inside a region of ``steps`` steps that starts on empty logs (uniform batch)."""
+    return steps // cap
+
+
+def graph_steps(cap: int) -> int:
     """Steps per captured graph: whole cycles that also return to the start of the token ring (in a
     staggered batch the list of rows to fold repeats with period cap as well)."""
-    import math
-
     return cap * Rig.RING // math.gcd(cap, Rig.RING)
+
+
+def segments(steps: int, seg: int):
+    """Split ``steps`` into ``(full segments of length seg, remainder)``."""
+    return steps // seg, steps % seg
 
 
 def capture_steps_with_merges_on_a_side_stream(rig: Rig, n_steps: int, main: "torch.cuda.Stream"):
@@ -311,36 +323,172 @@ def capture_steps_with_merges_on_a_side_stream(rig: Rig, n_steps: int, main: "to
     main.wait_event(join)
 
 
-def time_graph_loop(rig: Rig, steps: int):
-    """Time exactly ``steps`` steps replayed from one CUDA graph that holds ``graph_steps`` steps
-    (decode launches and the merge launches between them), the way a serving loop would run the
-    cycle.  ``steps`` must be a multiple of the graph length.  Returns total ms."""
-    g_len = graph_steps(rig.cap, rig.staggered)
-    assert steps % g_len == 0
-    stream = torch.cuda.Stream(device=rig.device)
-    graph = torch.cuda.CUDAGraph()
-    torch.cuda.synchronize()
+class Region:
+    """Enqueues EXACTLY ``steps`` steps of the hot path, starting from what ``reset_logs`` leaves.
+
+    With ``use_graph`` the steps are replayed from CUDA graphs the way a serving loop would run the
+    cycle: one graph of ``graph_steps(cap)`` steps (whole cycles that also return to the start of the
+    token ring) replayed ``steps // graph_steps`` times, and a second graph holding the remaining
+    ``steps % graph_steps`` steps; otherwise the steps are plain launches.  ``launches`` is the number of
+    kernels one pass over the region executes."""
+
+    def __init__(self, rig: Rig, steps: int, use_graph: bool):
+        self.rig, self.steps, self.use_graph = rig, steps, use_graph
+        self.stream = torch.cuda.Stream(device=rig.device)
+        self.plan, self.launches = [], None
+        if use_graph:
+            g_len = graph_steps(rig.cap)
+            n_full, tail = segments(steps, g_len)
+            self.launches = 0
+            for n, reps in ((g_len, n_full), (tail, 1)):
+                if n and reps:
+                    graph, count = self._capture(n)
+                    self.plan.append((graph, reps))
+                    self.launches += count * reps
+            self.describe = (f"CUDA graphs: {n_full} replay(s) of a {g_len}-step graph"
+                             + (f" + one {tail}-step graph" if tail else ""))
+        else:
+            self.describe = "plain launches"
+
+    def _capture(self, n):
+        rig, dl = self.rig, self.rig.dl
+        graph = torch.cuda.CUDAGraph()
+        rig.phase = 0     # every captured segment starts at the beginning of a cycle
+        torch.cuda.synchronize()
+        count0 = dl.launch_count()
+        with torch.cuda.stream(self.stream):
+            with torch.cuda.graph(graph, stream=self.stream):
+                if rig.overlap_merges:
+                    capture_steps_with_merges_on_a_side_stream(rig, n, self.stream)
+                else:
+                    for t in range(n):
+                        for layer in range(rig.layers):
+                            rig.step(t, layer)
+        rig.phase = 0
+        return graph, dl.launch_count() - count0   # the host-side counter sees the capture, not the replays
+
+    def enqueue(self):
+        """Called with ``self.stream`` current."""
+        rig = self.rig
+        if self.use_graph:
+            for graph, reps in self.plan:
+                for _ in range(reps):
+                    graph.replay()
+        else:
+            count0 = rig.dl.launch_count()
+            for t in range(self.steps):
+                for layer in range(rig.layers):
+                    rig.step(t, layer)
+            self.launches = rig.dl.launch_count() - count0
+
+
+def timed_passes(rig: Rig, enqueue, stream, clocks: "ClockSampler | None", device, reset=None):
+    """Time the region ``enqueue`` puts on ``stream``: logs emptied, barrier + synchronize, events on the
+    launching stream around the region, synchronize + barrier.  The first pass decides how often the
+    region is repeated (about TARGET_TIMED_MS in all, between MIN_REPEATS and MAX_REPEATS passes; the
+    count is taken from the maximum over ranks so that all ranks agree).  Returns the per-pass
+    milliseconds, each the maximum over ranks."""
+    reset = reset or rig.reset_logs
+    reset()                       # one untimed pass first: graph upload, instruction caches, clocks
     with torch.cuda.stream(stream):
-        with torch.cuda.graph(graph, stream=stream):
-            if rig.overlap_merges:
-                capture_steps_with_merges_on_a_side_stream(rig, g_len, stream)
-            else:
-                for t in range(g_len):
-                    for layer in range(rig.layers):
-                        rig.step(t, layer)
-        graph.replay()  # warm the replay path; a graph holds whole cycles, so every replay starts in the same phase
+        enqueue()
     torch.cuda.synchronize()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launch.barrier()
-    torch.cuda.synchronize()
-    with torch.cuda.stream(stream):
+    times = []
+    n_pass = MAX_REPEATS
+    while len(times) < n_pass:
+        reset()
+        torch.cuda.synchronize()
+        launch.barrier()
+        torch.cuda.synchronize()
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if clocks is not None:
+            clocks.busy = True
+        with torch.cuda.stream(stream):
+            start.record()
+            enqueue()
+            end.record()
+        torch.cuda.synchronize()
+        if clocks is not None:
+            clocks.busy = False
+        launch.barrier()
+        times.append(launch.max_over_ranks(start.elapsed_time(end), device))
+        if len(times) == 1:
+            n_pass = int(min(MAX_REPEATS, max(MIN_REPEATS, math.ceil(TARGET_TIMED_MS / max(times[0], 1e-3)))))
+    return times
+
+
+def time_kernel_split(rig: Rig, steps: int, passes: int = 3):
+    """The same K steps as plain launches with events that split the time into decode launches and
+    merge launches: one event pair around every run of consecutive decode launches (an event between
+    every pair of launches would itself cost several microseconds per step) and one around every
+    merge.  Returns ``(decode ms per launch, merge ms per launch or None, plain-launch ms per step)``,
+    each the median over ``passes`` passes."""
+    cap = rig.cap
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    dec_avg, mrg_avg, total = [], [], []
+    for _ in range(passes):
+        rig.reset_logs()
+        torch.cuda.synchronize()
+        start, end = ev(), ev()
+        runs, merges = [], []   # (event, event, decode launches between them), (event, event)
         start.record()
-        for _ in range(steps // g_len):
-            graph.replay()
+        for t in range(steps):
+            for layer in range(rig.layers):
+                mark = layer == 0   # one layer carries the events
+                if not mark:
+                    rig.step(t, layer)
+                    continue
+                if rig.staggered:   # per step: merge of the listed rows, then the decode launch
+                    a = ev(); a.record()
+                    rig.stag_merge(layer)
+                    b = ev(); b.record()
+                    rig.decode(t, layer)
+                    c = ev(); c.record()
+                    rig.end_layer(layer)
+                    if mark:
+                        merges.append((a, b))
+                        runs.append((b, c, 1))
+                    continue
+                if mark and t % cap == 0:
+                    a = ev(); a.record()
+                    run_start, run_n = a, 0
+                rig.decode(t, layer, chained=(rig.layers == 1 and t % cap != 0))
+                if mark:
+                    run_n += 1
+                last_of_run = (t + 1) % cap == 0 or t == steps - 1
+                if mark and last_of_run:
+                    b = ev(); b.record()
+                    runs.append((run_start, b, run_n))
+                if (t + 1) % cap == 0:
+                    rig.merge(layer)
+                    if mark:
+                        c = ev(); c.record()
+                        merges.append((b, c))
         end.record()
-    torch.cuda.synchronize()
-    launch.barrier()
-    return start.elapsed_time(end)
+        torch.cuda.synchronize()
+        dec_avg.append(sum(a.elapsed_time(b) for a, b, _ in runs) / sum(n for _, _, n in runs))
+        if merges:
+            mrg_avg.append(sum(a.elapsed_time(b) for a, b in merges) / len(merges))
+        total.append(start.elapsed_time(end) / steps)
+    return statistics.median(dec_avg), (statistics.median(mrg_avg) if mrg_avg else None), statistics.median(total)
+
+
+def time_merge_alone(rig: Rig, passes: int = 3):
+    """A merge of full logs on its own (uniform batch): used when the timed region holds no merge."""
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    res = []
+    for _ in range(passes):
+        rig.reset_logs()
+        for t in range(rig.cap):
+            rig.decode(t, 0)
+        a, b = ev(), ev()
+        torch.cuda.synchronize()
+        a.record()
+        rig.merge(0, only_if_full=False)
+        b.record()
+        torch.cuda.synchronize()
+        res.append(a.elapsed_time(b))
+    return statistics.median(res)
 
 
 def time_paper_cycle(rig: Rig, steps: int):
@@ -350,11 +498,10 @@ def time_paper_cycle(rig: Rig, steps: int):
     call sees slot -1 for the rows whose log is full, the fused-step call gets exactly those rows as
     its batch; the host knows each row's phase from its step counter, so the lists are precomputed for
     one period.
-    Timed as CUDA-graph replays of whole cycles; on a single-layer uniform batch the fused step alone
-    is then timed over plain launches with one event pair per cycle.
+    Timed as CUDA-graph replays of whole cycles (the step count is rounded to whole graphs, at least
+    one); on a single-layer uniform batch the fused step alone is then timed over plain launches with
+    one event pair per cycle.
     Returns (steps timed, total ms, mean ms of a fused-step launch or None)."""
-    import math
-
     cap, M = rig.cap, rig.cap + 1
     g_len = M * Rig.RING // math.gcd(M, Rig.RING)
     steps = max(steps // g_len, 1) * g_len
@@ -433,7 +580,9 @@ def time_paper_cycle(rig: Rig, steps: int):
 
 
 def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = True):
-    """The eager dense comparator on the same token ring, launched the same way as the main loop."""
+    """The eager dense comparator on the same token ring, launched the same way as the main loop (a
+    graph of one trip round the token ring, replayed; the step count is rounded to whole trips, at
+    least one).  Returns (steps timed, total ms)."""
     dl = rig.dl
 
     def launch_steps(n):
@@ -442,9 +591,9 @@ def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = Tru
             dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
                           u_bonus=rig.bonus[0], out=rig.out)
 
+    steps = max(steps // rig.RING, 2) * rig.RING
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    use_graph = use_graph and steps % rig.RING == 0
-    stream = torch.cuda.Stream(device=rig.device) if use_graph else torch.cuda.current_stream()
+    stream = torch.cuda.Stream(device=rig.device)
     graph = None
     torch.cuda.synchronize()
     with torch.cuda.stream(stream):
@@ -464,14 +613,15 @@ def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = Tru
             launch_steps(steps)
         end.record()
     torch.cuda.synchronize()
-    return start.elapsed_time(end)
+    return steps, start.elapsed_time(end)
 
 
-def time_e2e_loop(rig: Rig, steps: int, use_graph: bool = True):
-    """The same cycle through the host-buffer entry point: every step copies q, k, v, g, beta from
-    pinned host memory and reads the output back to pinned host memory.  Copy-in, kernel and
-    copy-out run on three streams over two staging sets (``deltalog_decode_step_host_overlapped``),
-    so the copies of step t+1 and t-1 overlap the kernel of step t."""
+def time_e2e(rig: Rig, steps: int, use_graph: bool, clocks, device):
+    """The same K steps through the host-buffer entry point: every step copies q, k, v, g, beta from
+    pinned host memory and reads the output back to pinned host memory.  Copy-in, kernel and copy-out
+    run on three streams over two staging sets (``deltalog_decode_step_host_overlapped``), so the copies
+    of step t+1 and t-1 overlap the kernel of step t.  The recurrent state stays resident (it is state,
+    not input).  Returns (per-pass ms, h2d bytes per step, d2h bytes per step, how it was launched)."""
     dl, wl = rig.dl, rig.wl
     streams = [torch.cuda.Stream(device=rig.device) for _ in range(3)]
     sets = [(dl.HostStaging(rig.desc, wl.batch, rig.device), dl.HostLane(*streams),
@@ -487,79 +637,84 @@ def time_e2e_loop(rig: Rig, steps: int, use_graph: bool = True):
             else:
                 host[k] = None
         host_ring.append(host)
-    rig.reset_logs()
-    torch.cuda.synchronize()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def run(n):
-        with torch.cuda.stream(streams[1]):  # merges go to the compute stream
-            if rig.staggered:
-                rig.merge(0)   # rows whose log is full fold before the first decode
+        """Steps 0..n-1 from freshly reset logs; merges go to the compute stream."""
+        with torch.cuda.stream(streams[1]):
             for t in range(n):
+                if rig.staggered:
+                    rig.merge(0)   # predicate merge: the rows whose log is full fold before the decode
                 tok = host_ring[t % rig.RING]
                 staging, lane, host_out = sets[t % 2]
                 dl.decode_step_host_overlapped(rig.desc, rig.states[0], staging, lane, tok["q"], tok["k"], tok["v"],
                                                tok["g"], tok["beta"], host_out, u_bonus=rig.bonus[0],
                                                slot_idx=rig.slot_idx)
-                if rig.staggered or (t + 1) % rig.cap == 0:
-                    rig.merge(0)   # predicate merge: after the step here, i.e. before the next decode
+                if not rig.staggered and (t + 1) % rig.cap == 0:
+                    rig.merge(0)
 
-    run(rig.cap)  # warm the copy path, ends on a merge
-    for st in streams:
-        st.synchronize()
-    # The serving-loop form: whole cycles of the three-stream pipeline (copies in, kernels, copies out,
-    # with their event dependencies) captured once into a CUDA graph through the same entry point and
-    # replayed; the host then only refills the pinned token buffers.  Falls back to plain calls.
-    import math
-    g_len = rig.cap * rig.RING // math.gcd(rig.cap, rig.RING)
-    graph = None
-    if use_graph and steps % g_len == 0 and not rig.staggered:
-        try:
-            graph = torch.cuda.CUDAGraph()
-            fork, j_in, j_out = torch.cuda.Event(), torch.cuda.Event(), torch.cuda.Event()
-            with torch.cuda.graph(graph, stream=streams[1]):
-                fork.record(streams[1])                      # bring the copy streams into the capture
-                streams[0].wait_event(fork)
-                streams[2].wait_event(fork)
-                for _, lane, _ in sets:                      # the lanes' events must belong to the capture
-                    lane.in_done.record(streams[0])
-                    lane.compute_done.record(streams[1])
-                    lane.out_done.record(streams[2])
-                run(g_len)
-                j_in.record(streams[0])
-                j_out.record(streams[2])
-                streams[1].wait_event(j_in)
-                streams[1].wait_event(j_out)
-            graph.replay()
-            torch.cuda.synchronize()
-        except Exception as exc:  # capture not possible here: time the plain calls instead
-            print(f"[bench] end-to-end graph capture failed ({type(exc).__name__}: {exc}); timing plain calls", file=sys.stderr)
-            graph = None
-            torch.cuda.synchronize()
-            rig.reset_logs()
-            torch.cuda.synchronize()
-    launch.barrier()
-    torch.cuda.synchronize()
-    if graph is not None:
-        with torch.cuda.stream(streams[1]):
-            start.record(streams[1])
-            for _ in range(steps // g_len):
-                graph.replay()
-            end.record(streams[1])
-    else:
-        start.record(streams[1])
-        run(steps)
+    def join_copy_streams():
+        j_in, j_out = torch.cuda.Event(), torch.cuda.Event()
+        j_in.record(streams[0])
+        j_out.record(streams[2])
+        streams[1].wait_event(j_in)
+        streams[1].wait_event(j_out)
+
+    def reset():
         for st in streams:
             st.synchronize()
-        end.record(streams[1])
-    torch.cuda.synchronize()
-    launch.barrier()
-    assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
+        rig.reset_logs()
+
+    reset()
+    run(min(steps, rig.cap))  # warm the copy path
+    for st in streams:
+        st.synchronize()
+    # The serving-loop form: the three-stream pipeline (copies in, kernels, copies out, with their event
+    # dependencies) captured into CUDA graphs through the same entry point and replayed, segmented like
+    # the device-resident region; the host then only refills the pinned token buffers.
+    plan, how = None, "plain calls"
+    if use_graph:
+        try:
+            g_len = graph_steps(rig.cap)
+            n_full, tail = segments(steps, g_len)
+            plan = []
+            for n, reps in ((g_len, n_full), (tail, 1)):
+                if not (n and reps):
+                    continue
+                graph = torch.cuda.CUDAGraph()
+                fork = torch.cuda.Event()
+                with torch.cuda.graph(graph, stream=streams[1]):
+                    fork.record(streams[1])                      # bring the copy streams into the capture
+                    streams[0].wait_event(fork)
+                    streams[2].wait_event(fork)
+                    for _, lane, _ in sets:                      # the lanes' events must belong to the capture
+                        lane.in_done.record(streams[0])
+                        lane.compute_done.record(streams[1])
+                        lane.out_done.record(streams[2])
+                    run(n)
+                    join_copy_streams()
+                plan.append((graph, reps))
+            how = (f"CUDA graphs: {n_full} replay(s) of a {g_len}-step graph" + (f" + one {tail}-step graph" if tail else ""))
+        except Exception as exc:  # capture not possible here: time the plain calls instead
+            print(f"[bench] end-to-end graph capture failed ({type(exc).__name__}: {exc}); timing plain calls", file=sys.stderr)
+            plan = None
+            torch.cuda.synchronize()
+
+    def enqueue():
+        if plan is not None:
+            for graph, reps in plan:
+                for _ in range(reps):
+                    graph.replay()
+        else:
+            run(steps)
+            join_copy_streams()
+
+    times = timed_passes(rig, enqueue, streams[1], clocks, device, reset=reset)
+    rig.check_status("end-to-end leg")
     staging = sets[0][0]
-    return start.elapsed_time(end), staging.h2d_bytes(rig.desc), staging.d2h_bytes()
+    return times, staging.h2d_bytes(rig.desc), staging.d2h_bytes(), how
 
 
-def cpu_baseline(wl, units: int, steps: int, chunk_units: int = 1024):
+def cpu_baseline(wl, units: int, steps: int, chunk_units: int = 1024, warmup: int = 0):
     """Time the fp64 oracle, as it stands, on a bounded sample of the workload's units.
 
     The sample is rolled through the oracle in chunks of ``chunk_units`` units (only the oracle
@@ -582,6 +737,9 @@ def cpu_baseline(wl, units: int, steps: int, chunk_units: int = 1024):
         q, k, v, g = f("q"), f("k"), f("v"), f("g")
         beta = f("beta")[..., 0] if wl.op != workloads.RWKV6 else None
         bon = np.tile(bonus.double().numpy(), (small.batch, 1)) if bonus is not None else None
+        if done == 0 and warmup > 0:   # untimed: pages the library in and starts the worker threads
+            w = min(warmup, steps)
+            oracle.eager_rollout(wl.op, S0, q[:w], k[:w], v[:w], g[:w], beta=beta[:w] if beta is not None else None, bonus=bon)
         t0 = time.perf_counter()
         oracle.eager_rollout(wl.op, S0, q, k, v, g, beta=beta, bonus=bon)
         dt += time.perf_counter() - t0
@@ -591,25 +749,63 @@ def cpu_baseline(wl, units: int, steps: int, chunk_units: int = 1024):
                       f"{dt:.2f} s on {oracle.num_threads()} threads"}, dt
 
 
-def run_reference(args, wl):
-    """``--impl reference``: the CPU oracle timed on the host cores (rank 0 only)."""
+def run_reference(args, wl, config_name):
+    """``--impl reference``: the CPU oracle timed on the host cores (rank 0 only; the other ranks leave
+    without work)."""
     rank, size, _ = launch.world()
     if rank != 0:
         return
-    units = 512 if args.steps <= 256 else 128   # bounds the fp64 input copies on the host (units x steps)
-    base, dt = cpu_baseline(wl, units, max(args.steps, 1))
+    steps = max(args.steps, 1)
+    units = 512 if steps <= 256 else 128   # bounds the fp64 input copies on the host (units x steps)
+    small = wl.scaled(layers=1)
+    base, dt = cpu_baseline(small, units, steps, warmup=max(args.warmup, 0))
     n_units = max(1, units // wl.H) * wl.H
     line = {
         "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "sample_units_per_step": n_units,
+        "config": {"workload": config_name, "sample_units_per_step": n_units,
                    "note": "each step is one token over a bounded sample of the workload's units on the host"},
         "cpu_baseline": {**base},
         "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+def dram_traffic(dl, config: int, cap: int, state: str):
+    """ncu DRAM bytes per launch for this configuration, or (None, why) when there is no capture of the
+    library build that is being timed."""
+    doc = ncu_traffic.load()
+    if not doc:
+        return None, "no profiles/dram_traffic.json"
+    if doc.get("build_id") != dl.build_id():
+        return None, f"profiles/dram_traffic.json is of build {doc.get('build_id')}, the library is build {dl.build_id()}"
+    cap_rec = doc.get("captures", {}).get(ncu_traffic.capture_key(config, cap, state))
+    if not cap_rec:
+        return None, "no capture of this configuration and capacity"
+    return cap_rec["kernels"], None
+
+
+def hot_loop_for_profilers(rig: Rig, args):
+    """``--only-hot-loop``: warm-up was done; run the steps as plain launches and leave."""
+    kind = args.hot_loop_kind
+    if kind == "cycle":
+        for t in range(args.steps):
+            for layer in range(rig.layers):
+                rig.step(t, layer)
+    elif kind == "eager":
+        S = rig.states[0].S_base
+        for t in range(args.steps):
+            tok = rig.rings[0][t % rig.RING]
+            rig.dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+                              u_bonus=rig.bonus[0], out=rig.out)
+    else:   # the paper's cycle: cap appends, then the fused merge step
+        M = rig.cap + 1
+        for t in range(args.steps):
+            (rig.fused if t % M == M - 1 else rig.decode)(t, 0)
+    torch.cuda.synchronize()
+    rig.check_status("hot loop")
 
 
 def main():
@@ -625,11 +821,16 @@ def main():
     ap.add_argument("--state", default="fp32", choices=["fp32", "bf16"],
                     help="dtype of the dense state; bf16 is the 16-bit-state variant (the configurations name fp32)")
     ap.add_argument("--only-hot-loop", action="store_true",
-                    help="warm-up and timed loop only (for profiler captures)")
+                    help="warm-up and then --steps steps as plain launches, nothing else (for profiler captures)")
+    ap.add_argument("--hot-loop-kind", default="cycle", choices=["cycle", "eager", "paper"],
+                    help="what --only-hot-loop runs: the decode/merge cycle, the eager kernel, or the paper's cycle")
     args = ap.parse_args()
+    if args.steps < 1:
+        ap.error("--steps must be at least 1")
     wl = workloads.CONFIGS[args.config]
+    config_name = f"configs[{args.config}] {wl.name}"
     if args.impl == "reference":
-        return run_reference(args, wl)
+        return run_reference(args, wl, config_name)
 
     rank, size, local = launch.init("nccl")
     assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
@@ -637,148 +838,186 @@ def main():
     device = torch.device("cuda", local)
     import paper_2608_15533_b200 as dl
 
-    cap = args.cap
+    cap, K = args.cap, args.steps
     warmup = max(args.warmup, 3)
     layers = wl.layers
     base16 = args.state == "bf16"
-    rig = Rig(wl, cap, device, seed_offset=rank, layers=layers, base16=base16)
+    # weak scaling: the global batch is `size` times the configuration's rows, sharded by rows
+    first_row, n_rows = launch.shard_rows(size * wl.batch, size, rank)
+    assert n_rows == wl.batch
+    rig = Rig(wl, cap, device, seed_offset=first_row // wl.batch, layers=layers, base16=base16)
     stag = rig.staggered
-    g_len = graph_steps(cap, stag)
     u = unit_shape(wl, base16=base16)
     units = wl.units
 
-    # ---- warm-up, then the timed region: exactly K steps ---------------------------------------
-    launches0 = dl.launch_count()
+    # ---- warm-up --------------------------------------------------------------------------------
     rig.reset_logs()
     for t in range(warmup):
         for layer in range(layers):
             rig.step(t, layer)
-    if not stag:
-        rig.reset_logs()   # a uniform batch starts the timed region on empty logs
     torch.cuda.synchronize()
-    warm_launches = dl.launch_count() - launches0
+    rig.check_status("warm-up")
     if args.only_hot_loop:
-        time_cycle_loop(rig, args.steps, per_kernel=False)
+        rig.reset_logs()
+        hot_loop_for_profilers(rig, args)
         return launch.finalize()
-    use_graph = (not args.no_graph) and args.steps % g_len == 0
+
+    # ---- the timed region: exactly K steps from empty logs, repeated, median ---------------------
+    use_graph = not args.no_graph
     with ClockSampler(local) as clocks:
-        l0 = dl.launch_count()
-        if use_graph:
-            total_ms = time_graph_loop(rig, args.steps)
-            # kernels executed by the replays (the host-side counter only sees the capture)
-            gpu_launches = layers * (2 * args.steps if stag else args.steps + args.steps // cap)
-        else:
-            total_ms, _, _, _ = time_cycle_loop(rig, args.steps, per_kernel=False)
-            gpu_launches = dl.launch_count() - l0
-        # same steps again as plain launches with two events per cycle: the split into decode and merge time
-        split_ms, dec_ms, mrg_ms, n_merges = time_cycle_loop(rig, args.steps)
-    assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
-    total_ms = launch.max_over_ranks(total_ms, device)
+        region = Region(rig, K, use_graph)
+        times = timed_passes(rig, region.enqueue, region.stream, clocks, device)
+        rig.check_status("timed region")
+        # the same steps as plain launches with events between the kernels: decode and merge time apart
+        clocks.busy = True
+        dec_ms, mrg_ms, plain_ms_per_step = time_kernel_split(rig, K)
+        merge_note = "merges of the timed region"
+        if mrg_ms is None:   # K < cap: the region holds no merge; time one on its own for the amortised figures
+            mrg_ms, merge_note = time_merge_alone(rig), "no merge falls into the timed region; a merge of full logs timed on its own"
+        clocks.busy = False
+        rig.check_status("per-kernel pass")
+        # ---- end-to-end leg: token tensors from pinned host memory, output back to the host ----------
+        e2e_times, h2d, d2h, e2e_how = time_e2e(rig, K, use_graph, clocks, device)
+    total_ms = statistics.median(times)
     all_units = launch.sum_over_ranks(units * layers, device)
-    ms_per_step = total_ms / args.steps
-    value = all_units * args.steps / (total_ms * 1e-3)
+    ms_per_step = total_ms / K
+    value = all_units * K / (total_ms * 1e-3)
+    n_merges = (K * layers) if stag else merges_in(K, cap) * layers
 
     cyc = traffic.cycle_bytes(u, cap)
     peak, peak_kind = measured_peak_gbs()
-    fills = [t % cap for t in range(args.steps)]
-    dec_bytes = statistics.mean(traffic.decode_read(u, f) + traffic.decode_write(u) for f in fills) * units
-    # events bracket cap decode launches per mark in a uniform batch, one decode launch per mark in a staggered one
-    dec_ms_avg = dec_ms / (n_merges * (1 if stag else cap)) if n_merges else float("nan")
-    achieved = dec_bytes / (dec_ms_avg * 1e-3) / 1e9
-    traffic_ncu = None if base16 else NCU_DECODE_TRAFFIC_PER_UNIT.get((args.config, cap))
+    if stag:   # fills uniform on 0..cap-1 across the rows at every step
+        dec_bytes = statistics.mean(traffic.decode_read(u, f) + traffic.decode_write(u) for f in range(cap)) * units
+    else:
+        dec_bytes = statistics.mean(traffic.decode_read(u, t % cap) + traffic.decode_write(u) for t in range(K)) * units
+    algo_gbs = dec_bytes / (dec_ms * 1e-3) / 1e9
+    kernels, why_not = dram_traffic(dl, args.config, cap, args.state)
+    dec_traffic = mrg_traffic = None
+    if kernels and "decode" in kernels:
+        dec_traffic = kernels["decode"]["dram_read_bytes_per_launch"] + kernels["decode"]["dram_write_bytes_per_launch"]
+    if kernels and "merge" in kernels:
+        mrg_traffic = kernels["merge"]["dram_read_bytes_per_launch"] + kernels["merge"]["dram_write_bytes_per_launch"]
+    dram_gbs = dec_traffic / (dec_ms * 1e-3) / 1e9 if dec_traffic else None
+    achieved = dram_gbs if dram_gbs is not None else algo_gbs
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": args.steps, "warmup": warmup,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": size, "steps": K, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {
-            "workload": f"configs[{args.config}] {wl.name}", "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
+            "workload": config_name, "op": workloads.OP_NAMES[wl.op], "batch": wl.batch,
             "H": wl.H, "d_k": wl.d, "d_v": wl.d, "layers": layers, "log_capacity": cap, "state": args.state,
-            "io": str(wl.io_dtype).replace("torch.", ""), "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1"
+            "io": str(wl.io_dtype).replace("torch.", ""),
+            "merge": ("before every step the rows whose log is full (listed by the host from its step counters) are folded; fills staggered over 0..cap-1"
                       + ("; the merges run on a side stream, overlapped with other layers' decode steps" if rig.overlap_merges and use_graph else "") if stag
                       else f"after every {cap}th step"),
-            "launch": (f"one CUDA graph of {g_len} steps, replayed" if use_graph else "plain launches"),
+            "merges_in_timed_region": n_merges,
+            "timed_region": f"exactly {K} steps from empty logs; repeated {len(times)} times (logs emptied in between, untimed), median reported",
+            "timed_region_ms_all": [round(x, 4) for x in times],
+            "launch": region.describe,
             "l2": f"inputs larger than L2: {units * u.state * layers / 2**20:.0f} MiB of base state per step, no flush",
-            "parallelism": f"rows sharded over {size} GPU(s), no collective",
+            "parallelism": f"global batch of {size * wl.batch} rows sharded by rows over {size} GPU(s), no collective",
         },
         "clocks": clocks.summary(),
-        "gpu_launches": gpu_launches,
+        "gpu_launches": region.launches,
         "roofline": {
-            "bound": "hbm", "kernel": "decode_pipelined_kernel" if wl.d == 128 else "decode_append_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-            "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic_ncu * units if traffic_ncu else None,
-            "traffic_note": ("ncu --cache-control none (L2 as the previous launch left it, as in the timed loop): base tiles are "
-                             "read evict-first, so part of the live log is served by L2 and DRAM traffic is below the "
-                             "algorithmic bytes that `achieved` counts"),
-            "algorithmic_bytes_per_launch": dec_bytes, "avg_launch_ms": dec_ms_avg,
+            "bound": "hbm", "kernel": "decode_pipelined_kernel" if wl.d == 128 else "decode_append_kernel",
+            "achieved": achieved, "achieved_kind": "dram bytes (ncu) / launch time" if dram_gbs is not None else "algorithmic bytes / launch time (no ncu capture of this build)",
+            "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+            "traffic": dec_traffic, "traffic_unavailable": why_not,
+            "traffic_note": ("dram__bytes_read.sum + dram__bytes_write.sum per launch, mean over the launches of a cycle, ncu "
+                             "--cache-control none (L2 as the previous launch left it, as in the timed loop): base tiles are "
+                             "read evict-first and the live log is kept in L2, so DRAM traffic is below the algorithmic bytes"),
+            "algorithmic_bytes_per_launch": dec_bytes, "avg_launch_ms": dec_ms,
+            "achieved_algorithmic_incl_l2": algo_gbs, "frac_algorithmic_incl_l2": algo_gbs / peak,
             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         },
-        "amortized": {
-            "algorithmic_bytes_per_unit_step": cyc["total"],
-            "hbm_gbs": cyc["total"] * all_units / (ms_per_step * 1e-3) / 1e9,
-            "bytes_written_per_unit_step": cyc["write"], "write_reduction_vs_eager": cyc["write_reduction"],
-            "decode_ms_per_step": dec_ms_avg, "merge_ms_per_merge": (mrg_ms / n_merges) if n_merges else None,
-            "plain_launch_ms_per_step": split_ms / args.steps,
-        },
     }
-    line["amortized"]["frac_of_nominal_8TBs"] = line["amortized"]["hbm_gbs"] / NOMINAL_HBM_GBS / size
-    line["amortized"]["frac_of_measured"] = line["amortized"]["hbm_gbs"] / peak / size
+    # amortised over a whole cycle from the per-kernel times: cap decode launches + one merge
+    if stag:
+        cycle_ms_per_step = (dec_ms + mrg_ms) * layers
+    else:
+        cycle_ms_per_step = dec_ms + mrg_ms / cap
+    am = {
+        "algorithmic_bytes_per_unit_step": cyc["total"],
+        "algorithmic_gbs_incl_l2": cyc["total"] * units * layers / (cycle_ms_per_step * 1e-3) / 1e9,
+        "bytes_written_per_unit_step": cyc["write"], "write_reduction_vs_eager": cyc["write_reduction"],
+        "decode_ms_per_launch": dec_ms, "merge_ms_per_launch": mrg_ms, "merge_time_from": merge_note,
+        "cycle_ms_per_step_from_kernel_times": cycle_ms_per_step, "plain_launch_ms_per_step": plain_ms_per_step,
+    }
+    am["algorithmic_frac_of_nominal_8TBs"] = am["algorithmic_gbs_incl_l2"] / NOMINAL_HBM_GBS
+    am["algorithmic_frac_of_measured"] = am["algorithmic_gbs_incl_l2"] / peak
+    if dec_traffic and mrg_traffic and not stag:
+        per_step = dec_traffic + mrg_traffic / cap
+        am["dram_bytes_per_unit_step"] = per_step / units
+        am["dram_gbs"] = per_step / (cycle_ms_per_step * 1e-3) / 1e9
+        am["dram_frac_of_measured"] = am["dram_gbs"] / peak
+        am["dram_frac_of_nominal_8TBs"] = am["dram_gbs"] / NOMINAL_HBM_GBS
+        am["dram_bytes_written_per_unit_step"] = (kernels["decode"]["dram_write_bytes_per_launch"]
+                                                  + kernels["merge"]["dram_write_bytes_per_launch"] / cap) / units
+        if "eager" in kernels:
+            am["dram_bytes_written_per_unit_step_eager"] = kernels["eager"]["dram_write_bytes_per_launch"] / units
+            am["dram_write_reduction_vs_eager"] = (am["dram_bytes_written_per_unit_step_eager"]
+                                                   / am["dram_bytes_written_per_unit_step"])
+    line["amortized"] = am
 
-    # ---- end-to-end leg: token tensors from pinned host memory, output back to the host --------
-    e2e_ms, h2d, d2h = time_e2e_loop(rig, args.steps, use_graph)
-    e2e_ms = launch.max_over_ranks(e2e_ms, device)
+    e2e_ms = statistics.median(e2e_times)
     e2e_units = launch.sum_over_ranks(units, device)
-    line["e2e"] = {"value": e2e_units * args.steps / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                   "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps,
+    line["e2e"] = {"value": e2e_units * K / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                   "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / K, "launch": e2e_how, "repeats": len(e2e_times),
                    "note": "state stays resident; q,k,v,g,beta in and out back every step, layer 0"}
 
     if not args.no_extras and rank == 0:
         # eager dense comparator on the same inputs
         rig.reset_logs()
         S = rig.states[0].S_base
-        eager_ms = time_eager_loop(rig, S, args.steps, use_graph) / args.steps
+        e_steps, e_total = time_eager_loop(rig, S, K, use_graph)
+        eager_ms = e_total / e_steps
         eager_bytes = (traffic.eager_read(u) + traffic.eager_write(u)) * units
-        line["eager_kernel"] = {"ms_per_step": eager_ms, "value": units / (eager_ms * 1e-3),
-                                "hbm_gbs": eager_bytes / (eager_ms * 1e-3) / 1e9,
+        line["eager_kernel"] = {"ms_per_step": eager_ms, "value": units / (eager_ms * 1e-3), "steps": e_steps,
+                                "algorithmic_gbs": eager_bytes / (eager_ms * 1e-3) / 1e9,
                                 "bytes_written_per_unit_step": traffic.eager_write(u)}
-        line["speedup_vs_eager_kernel"] = eager_ms / (ms_per_step / layers)
+        line["speedup_vs_eager_kernel"] = eager_ms / (cycle_ms_per_step / layers)
         # the paper's own cycle: cap appends + one fused merge step (cap + 1 tokens per dense write)
-        p_steps, p_ms, fused_ms = time_paper_cycle(rig, args.steps)
+        p_steps, p_ms, fused_ms = time_paper_cycle(rig, K)
         pc = traffic.paper_cycle_bytes(u, cap + 1)
         p_step_ms = p_ms / p_steps
         line["paper_cycle"] = {
             "ms_per_step": p_step_ms, "value": units * layers * p_steps / (p_ms * 1e-3), "steps": p_steps,
             "merge_interval_M": cap + 1, "algorithmic_bytes_per_unit_step": pc["total"],
-            "hbm_gbs": pc["total"] * units * layers / (p_step_ms * 1e-3) / 1e9,
+            "algorithmic_gbs_incl_l2": pc["total"] * units * layers / (p_step_ms * 1e-3) / 1e9,
             "launch": ("two launches per layer-step over phase-split batches" if stag else "one launch per step"),
             "speedup_vs_eager_kernel": eager_ms / (p_step_ms / layers)}
         if fused_ms is not None:
             fused_bytes = (traffic.fused_read(u, cap) + traffic.fused_write(u)) * units
             line["paper_cycle"]["fused_step_ms"] = fused_ms
-            line["paper_cycle"]["fused_step_hbm_gbs"] = fused_bytes / (fused_ms * 1e-3) / 1e9
-        assert all(s == 0 for s in rig.status()), f"device status bits set: {rig.status()}"
+            line["paper_cycle"]["fused_step_algorithmic_gbs"] = fused_bytes / (fused_ms * 1e-3) / 1e9
+        rig.check_status("paper cycle")
+        # capacity sweep: whole cycles (at least 32 steps' worth), write reduction per capacity
         sweep = {}
-        for c in wl.caps:
-            if c == cap and layers == 1:
-                sweep[str(c)] = {"ms_per_step": ms_per_step, "value": value,
-                                 "write_reduction_vs_eager": cyc["write_reduction"],
-                                 "hbm_gbs": line["amortized"]["hbm_gbs"]}
-                continue
+        for c in ([cap] if cap in wl.caps else []) + [c for c in wl.caps if c != cap]:   # the rig at hand first
             if layers > 1:
                 continue
-            del rig
-            torch.cuda.empty_cache()
-            rig = Rig(wl, c, device, seed_offset=rank, base16=base16)
-            for t in range(max(c, 3)):
-                rig.decode(t);
-                if (t + 1) % c == 0:
-                    rig.merge()
-            rig.reset_logs()
-            ms = time_graph_loop(rig, args.steps) if use_graph and args.steps % graph_steps(c) == 0 else \
-                time_cycle_loop(rig, args.steps, per_kernel=False)[0]
             cc = traffic.cycle_bytes(u, c)
-            sweep[str(c)] = {"ms_per_step": ms / args.steps, "value": units * args.steps / (ms * 1e-3),
+            n = max(K // graph_steps(c), max(1, 32 // graph_steps(c))) * graph_steps(c)   # whole graphs
+            if c == cap and n == K:
+                ms = ms_per_step
+            else:
+                if c != cap:
+                    del rig
+                    torch.cuda.empty_cache()
+                    rig = Rig(wl, c, device, seed_offset=first_row // wl.batch, base16=base16)
+                    for t in range(max(c, 3)):
+                        rig.step(t)
+                sweep_region = Region(rig, n, use_graph)
+                ms = statistics.median(timed_passes(rig, sweep_region.enqueue, sweep_region.stream, None, device)) / n
+                rig.check_status(f"capacity sweep, cap {c}")
+            sweep[str(c)] = {"ms_per_step": ms, "value": units / (ms * 1e-3),
+                             "bytes_written_per_unit_step": cc["write"],
                              "write_reduction_vs_eager": cc["write_reduction"],
-                             "hbm_gbs": cc["total"] * units / (ms / args.steps * 1e-3) / 1e9}
-        line["capacity_sweep"] = sweep
+                             "algorithmic_gbs_incl_l2": cc["total"] * units / (ms * 1e-3) / 1e9}
+        if sweep:
+            line["capacity_sweep"] = sweep
+            line["capacity_sweep_note"] = "whole cycles per capacity (steps rounded to whole graphs); bytes from the byte model"
         small = wl.scaled(layers=1)
         line["cpu_baseline"], _ = cpu_baseline(small, min(wl.units, 4096), 128)
     if rank == 0:

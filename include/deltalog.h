@@ -97,17 +97,26 @@ typedef struct {
 } deltalog_desc;
 
 /*
- * Hints (deltalog_desc.hints).  A hint is a promise by the caller; breaking it is a data race.
+ * Hints (deltalog_desc.hints).  A hint is a promise by the caller; breaking it is a data race.  The paper
+ * has no counterpart; the hints remove the ramp-up and tail of back-to-back decode launches (a few
+ * microseconds each).
  *   DELTALOG_HINT_BASE_UNTOUCHED  The work queued on the stream directly in front of this
- *       deltalog_decode_step does not write S_base of the slots this call reads (it was another
- *       decode step on this state, or unrelated work -- NOT a deltalog_merge, deltalog_decode_merge_step,
- *       deltalog_reset_slots or deltalog_eager_step on these slots).  The decode kernel is then
- *       launched with programmatic stream serialisation: its CTAs start while the preceding kernel is
- *       still retiring and stream base tiles at once; lengths, log entries and everything else are
- *       read only after the preceding kernel has completed.  The paper has no counterpart; it removes the
- *       ramp-up and tail of back-to-back decode launches (a few microseconds each).
+ *       deltalog_decode_step does not WRITE S_base of the slots this call reads.  (True when it was
+ *       another decode step on this state, or the kernel that produced this step's q, k, v, g, beta;
+ *       NOT true for deltalog_merge, deltalog_decode_merge_step, deltalog_reset_slots or
+ *       deltalog_eager_step on these slots.)  The decode kernel is then launched with programmatic
+ *       stream serialisation: its CTAs may start while the preceding kernel is still retiring.  Ahead of
+ *       that kernel's completion they read base tiles and nothing else -- unless the next hint allows the
+ *       slot list too.  Everything else this call reads (q, k, v, g, beta, u_bonus, lengths, log
+ *       entries) is read only after the preceding kernel has completed and its writes are visible, so
+ *       the preceding kernel may well be the one that writes those tensors.
+ *   DELTALOG_HINT_SLOTS_STABLE    In addition: the work directly in front does not write slot_idx
+ *       either.  Base tiles are addressed through slot_idx, so with a non-NULL slot_idx the early start
+ *       above streams tiles only under this second promise; without it the kernel still overlaps its
+ *       launch latency with the preceding kernel but waits before its first read.  With slot_idx == NULL
+ *       the bit changes nothing.
  */
-enum { DELTALOG_HINT_BASE_UNTOUCHED = 1 };
+enum { DELTALOG_HINT_BASE_UNTOUCHED = 1, DELTALOG_HINT_SLOTS_STABLE = 2 };
 
 /* Physical state (Section 3.1).  Device pointers, caller-owned. d_lambda = 1 (GDN) or d_k. */
 typedef struct {
@@ -289,6 +298,11 @@ const char *deltalog_status_string(int code);
 
 /* Library version, major * 10000 + minor * 100 + patch. */
 int deltalog_version(void);
+
+/* Identifier of the sources and compiler switches this library was built from (static storage; "unknown"
+ * when the build did not supply one).  Profiler figures stored beside the code carry the identifier of the
+ * build they were captured on. */
+const char *deltalog_build_id(void);
 
 /* Number of kernels the library has launched in this process (host counter, all entry points). */
 uint64_t deltalog_launch_count(void);

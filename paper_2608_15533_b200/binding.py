@@ -15,7 +15,7 @@ from typing import Optional
 import torch
 
 GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
-HINT_BASE_UNTOUCHED = 1
+HINT_BASE_UNTOUCHED, HINT_SLOTS_STABLE = 1, 2
 _DELTA_RULE = (GDN, KDA)            # b = beta (v - S'^T k): U log in fp32
 _VEC_DECAY = (KDA, RWKV6, GLA)      # one log-decay per key channel
 F32, BF16 = 0, 1
@@ -31,7 +31,7 @@ LIB_PATH = Path(__file__).resolve().parent / "libdeltalog.so"
 EXPORTS = (
     "deltalog_decode_step", "deltalog_decode_steps", "deltalog_decode_merge_step", "deltalog_merge", "deltalog_reset_slots", "deltalog_eager_step", "deltalog_decode_step_host",
     "deltalog_decode_step_host_static", "deltalog_decode_step_host_overlapped",
-    "deltalog_status_string", "deltalog_version", "deltalog_launch_count",
+    "deltalog_status_string", "deltalog_version", "deltalog_build_id", "deltalog_launch_count",
 )
 
 
@@ -96,6 +96,7 @@ def load_library() -> ctypes.CDLL:
         lib.deltalog_status_string.restype = ctypes.c_char_p
         lib.deltalog_status_string.argtypes = [ctypes.c_int]
         lib.deltalog_version.restype = ctypes.c_int
+        lib.deltalog_build_id.restype = ctypes.c_char_p
         lib.deltalog_launch_count.restype = ctypes.c_uint64
         _lib = lib
     return _lib
@@ -107,6 +108,11 @@ def status_string(code: int) -> str:
 
 def version() -> int:
     return int(load_library().deltalog_version())
+
+
+def build_id() -> str:
+    """Identifier of the sources the loaded library was built from (see ``build.source_id``)."""
+    return load_library().deltalog_build_id().decode()
 
 
 def launch_count() -> int:

@@ -31,6 +31,25 @@ def sources():
     return sorted(CSRC.glob("*.cu"))
 
 
+def extra_flags():
+    """Extra compiler switches for experiments (``DELTALOG_NVCC_EXTRA="-D..."``)."""
+    return os.environ.get("DELTALOG_NVCC_EXTRA", "").split()
+
+
+def source_id(extra=()) -> str:
+    """Twelve hex digits identifying what the library is built from: every file under ``csrc/``, the
+    header and the compiler switches.  It is compiled into the library (``deltalog_build_id``), and
+    profiler figures kept beside the code carry it, so a figure taken from another build is recognised."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for path in sorted(list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(INCLUDE.glob("*.h"))):
+        h.update(path.name.encode())
+        h.update(path.read_bytes())
+    h.update(" ".join([*NVCC_FLAGS, *extra]).encode())
+    return h.hexdigest()[:12]
+
+
 def _stale() -> bool:
     if not LIB.exists():
         return True
@@ -44,8 +63,9 @@ def build_library(force: bool = False, verbose: bool = False) -> Path:
     if not force and not _stale():
         return LIB
     tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    extra = os.environ.get("DELTALOG_NVCC_EXTRA", "").split()  # extra -D switches for experiments
-    cmd = [_nvcc(), *NVCC_FLAGS, *extra, f"-I{INCLUDE}", f"-I{CSRC}", *map(str, sources()), "-o", str(tmp)]
+    extra = extra_flags()
+    cmd = [_nvcc(), *NVCC_FLAGS, *extra, f'-DDELTALOG_BUILD_ID="{source_id(extra)}"', f"-I{INCLUDE}", f"-I{CSRC}",
+           *map(str, sources()), "-o", str(tmp)]
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode != 0:
         sys.stderr.write(proc.stdout + proc.stderr)

@@ -58,6 +58,9 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    // Chained launch (see DELTALOG_HINT_BASE_UNTOUCHED): the slot list is read ahead of the preceding
+    // kernel's completion only if there is none or the caller vouched for it (DELTALOG_HINT_SLOTS_STABLE).
+    if (tk.slot_idx != nullptr && !(tk.hints & DELTALOG_HINT_SLOTS_STABLE)) asm volatile("griddepcontrol.wait;\n" ::: "memory");
     int slot;
     if (!resolve_slot(tk.slot_idx, b, st.num_slots, st.status, tid, slot)) return;
     const size_t unit = (size_t)slot * st.H + h;  // (slot, head) in the state pool
@@ -78,7 +81,7 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
     const int len = st.log_len[unit];
-    if (len >= cap) {  // Algorithm 1's else-branch is the caller's job (deltalog_merge)
+    if (len >= cap || len < 0) {  // full: Algorithm 1's else-branch is the caller's job (deltalog_merge); < 0: corrupt
         if (tid == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_LOG_FULL);
         return;
     }

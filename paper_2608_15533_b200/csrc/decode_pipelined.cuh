@@ -47,7 +47,18 @@ constexpr int kBaseWarps = 4;                          // base-ring producer war
 #endif
 constexpr int kAuxWarps = DELTALOG_AUX_WARPS;          // aux-ring producer warps: they take the units in turn
 constexpr int kPipeThreads = 2 * kPipeConsumers + 32 * (kBaseWarps + kAuxWarps);  // + base and aux producers
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+// Upper bound on any single wait inside the kernel (compile-time knob; the give-up path is exercised by a
+// test build with a limit of a few milliseconds).
+#ifndef DELTALOG_WAIT_LIMIT_NS
+#define DELTALOG_WAIT_LIMIT_NS 2000000000ull  // 2 s per wait
+#endif
+constexpr unsigned long long kWaitLimitNs = DELTALOG_WAIT_LIMIT_NS;
+// Test builds only (-DDELTALOG_TEST_HOOKS=1): PipeCfg.test_drop_item names one unit (global index) whose
+// chunk 0 the base producer never requests, so that the stream group's wait for it runs out -- the only
+// way to see the give-up path of the bounded waits without hanging or faulting anything.
+#ifndef DELTALOG_TEST_HOOKS
+#define DELTALOG_TEST_HOOKS 0
+#endif
 
 enum : int { kMetaSkip = 1, kMetaFull = 2 };
 
@@ -92,6 +103,7 @@ struct PipeCfg {
     int n_base;  // stages of the base ring
     int n_aux;   // stages of the aux ring
     int slot_shift;  // log2 of the number of hand-over slots (1 or 2)
+    int test_drop_item;  // -1; a unit index only in test builds (DELTALOG_TEST_HOOKS)
 };
 
 template <int OP, int D, typename IO, typename UL, typename BT = float>
@@ -260,6 +272,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
 
     const int total = tk.B * st.H;
+    const bool slots_early = tk.slot_idx == nullptr || (tk.hints & DELTALOG_HINT_SLOTS_STABLE) != 0;
     const int first = blockIdx.x, stride = gridDim.x;
     const int n_items = (total - first + stride - 1) / stride;
     const int cap = st.cap, H = st.H;
@@ -286,6 +299,11 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         // stay: what L2 can hold beside the log need not be fetched from HBM again by the next step
         const float pin_fraction = fminf(1.f, st.l2_pin_bytes / ((float)total * (float)(D * D) * (float)sizeof(BT)));
         const uint64_t stream_policy = pin_fraction > 0.f ? l2_policy_keep(pin_fraction) : l2_policy_evict_first();
+        // Started ahead of the preceding kernel's completion (chained launch), these warps read two things
+        // early: the slot list and the base tiles.  The caller vouched for the tiles
+        // (DELTALOG_HINT_BASE_UNTOUCHED); the slot list may be read early only if there is none or the
+        // caller vouched for it as well (DELTALOG_HINT_SLOTS_STABLE) -- otherwise wait here.
+        if (!slots_early) asm volatile("griddepcontrol.wait;\n" ::: "memory");
         for (int it0 = 0; it0 < n_items && c < NCHUNK; it0 += 32) {
             int slot = -1;
             if (it0 + lane < n_items) {
@@ -297,6 +315,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             for (int j = 0; j < cnt; ++j) {
                 const int s = __shfl_sync(0xffffffffu, slot, j);
                 if (s < 0) continue;
+#if DELTALOG_TEST_HOOKS
+                if (c == 0 && first + (it0 + j) * stride == cfg.test_drop_item) dead = true;  // never requested
+#endif
                 if (lane == 0 && !dead) {
                     const int h = (first + (it0 + j) * stride) % H;
                     const char *src = static_cast<const char *>(st.S_base) + ((size_t)s * H + h) * D * D * sizeof(BT);
@@ -339,12 +360,17 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         bool dead = false;
         int n_done = 0;  // own units queued so far
         const int io_vec = D * (int)sizeof(IO);
-        // Lengths and log entries are written by the step before this one: when this kernel was
-        // launched ahead of the previous kernel's completion, wait for it before the first length is
-        // read (a no-op otherwise) -- after the slot indices and the per-unit token scalars, which are
-        // inputs, have been requested.  Everything the other roles do with global memory follows from
-        // what these warps load.
+        // Lengths and log entries are written by the step before this one, and the token tensors
+        // (gate, beta, q, k, v) are typically produced by the launch directly in front of this one: when
+        // this kernel was started ahead of the previous kernel's completion, wait for it before any of
+        // them is read (a no-op otherwise).  Only the slot indices are requested before the wait, and only
+        // when the caller vouched for them.  Everything the other roles do with global memory follows
+        // from what these warps load.
         bool waited = false;
+        if (!slots_early) {
+            asm volatile("griddepcontrol.wait;\n" ::: "memory");
+            waited = true;
+        }
         for (int n0 = 0; a + kAuxWarps * n0 < n_items; n0 += 32) {
             int slot = -1, len = 0, flags = kMetaSkip, item = 0;
             float gs = 0.f, bt = 0.f;
@@ -356,16 +382,14 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     if (st.status) atomicOr(st.status, DELTALOG_STATUS_BAD_SLOT);
                     slot = -1;
                 }
-                if (slot >= 0) {
-                    if (!kVecDecay && tk.g) gs = tk.g[item];  // no gate: plain linear attention
-                    if (kDelta) bt = tk.beta[item];
-                }
             }
             if (!waited) {
                 asm volatile("griddepcontrol.wait;\n" ::: "memory");
                 waited = true;
             }
             if (slot >= 0) {
+                if (!kVecDecay && tk.g) gs = tk.g[item];  // no gate: plain linear attention
+                if (kDelta) bt = tk.beta[item];
                 len = st.log_len[(size_t)slot * H + item % H];
                 flags = 0;
                 if (len >= cap || len < 0) {

@@ -16,60 +16,12 @@
 #include "fused_step_kernel.cuh"
 #include "merge_kernel.cuh"
 #include "merge_tc_kernel.cuh"
+#include "validate.h"
 
 namespace deltalog {
 namespace {
 
 std::atomic<uint64_t> g_launches{0};
-
-bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-// Operator facts needed on the host side (Table 1).
-bool op_delta_rule(int op) { return op == DELTALOG_GDN || op == DELTALOG_KDA; }
-bool op_has_gate(int op) { return op != DELTALOG_LINATTN; }
-bool op_vec_decay(int op) { return op == DELTALOG_KDA || op == DELTALOG_RWKV6 || op == DELTALOG_GLA; }
-
-int validate_desc(const deltalog_desc *d) {
-    if (!d) return DELTALOG_ERR_INVALID_ARG;
-    if (d->op < DELTALOG_GDN || d->op > DELTALOG_GLA) return DELTALOG_ERR_INVALID_ARG;
-    if (d->num_slots <= 0 || d->H <= 0) return DELTALOG_ERR_INVALID_ARG;
-    if (d->H_qk < 0 || (d->H_qk > 0 && d->H % d->H_qk != 0)) return DELTALOG_ERR_INVALID_ARG;
-    if (d->io_dtype != DELTALOG_F32 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
-    if (d->klog_dtype != DELTALOG_F32 && d->klog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
-    if (d->ulog_dtype != DELTALOG_F32 && d->ulog_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
-    if (d->d_k != d->d_v || (d->d_k != 64 && d->d_k != 128)) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    if (d->klog_dtype != d->io_dtype) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    // b = v is lossless in the I/O dtype; the delta rule keeps b in fp32 unless the caller asks for the
-    // reduced-precision 16-bit U log (only with 16-bit I/O)
-    const bool u_ok = op_delta_rule(d->op) ? (d->ulog_dtype == DELTALOG_F32 || d->ulog_dtype == d->io_dtype)
-                                           : d->ulog_dtype == d->io_dtype;
-    if (!u_ok) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    if (d->cap < 1 || d->cap > kMaxCap) return DELTALOG_ERR_CAP_RANGE;
-    if (d->base_dtype != DELTALOG_F32 && d->base_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
-    // the 16-bit dense state is built for the 16-bit I/O configurations only
-    if (d->base_dtype == DELTALOG_BF16 && d->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_UNSUPPORTED_SHAPE;
-    return DELTALOG_OK;
-}
-
-int validate_state(const deltalog_state *s) {
-    if (!s || !s->S_base || !s->K_log || !s->U_log || !s->decay_log || !s->log_len)
-        return DELTALOG_ERR_INVALID_ARG;
-    if (!aligned16(s->S_base) || !aligned16(s->K_log) || !aligned16(s->U_log) || !aligned16(s->decay_log))
-        return DELTALOG_ERR_INVALID_ARG;
-    return DELTALOG_OK;
-}
-
-int validate_token(const deltalog_desc *d, const void *q, const void *k, const void *v, const float *g,
-                   const float *beta, const float *u_bonus, int32_t B, const void *out) {
-    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
-    if (!q || !k || !v || !out) return DELTALOG_ERR_INVALID_ARG;
-    if (op_has_gate(d->op) && !g) return DELTALOG_ERR_INVALID_ARG;
-    if (op_delta_rule(d->op) && !beta) return DELTALOG_ERR_INVALID_ARG;
-    if (d->op == DELTALOG_RWKV6 && !u_bonus) return DELTALOG_ERR_INVALID_ARG;
-    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || (op_has_gate(d->op) && !aligned16(g)))
-        return DELTALOG_ERR_INVALID_ARG;
-    return DELTALOG_OK;
-}
 
 int qk_heads(const deltalog_desc *d) { return d->H_qk > 0 ? d->H_qk : d->H; }
 
@@ -114,6 +66,9 @@ int env_int(const char *name, int dflt) {
     const char *v = std::getenv(name);
     return v ? std::atoi(v) : dflt;
 }
+#if DELTALOG_TEST_HOOKS
+int env_int_now(const char *name, int dflt) { return env_int(name, dflt); }  // read at every launch
+#endif
 
 StateArgs make_state_args(const deltalog_desc *d, const deltalog_state *s) {
     StateArgs a;
@@ -221,10 +176,14 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
     // more than they hide, so the one-CTA-per-unit kernel is the faster one there (measured).
     bool pipelined = impl != 1 && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0) && (D == 128 || impl == 2);
     constexpr int kStage = chunk_bytes<D, BT>();
+    constexpr int kChunks = D * D * (int)sizeof(BT) / kStage;  // chunks per base tile
     // hand-over slots: two while the base tile's arrival sets the pace; with a 16-bit base the chain
     // prep -> stream -> epilogue is the longer one and four units are kept in flight
     static const int env_slots = env_int("DELTALOG_PIPE_SLOTS", 0);
-    PipeCfg cfg{0, 0, env_slots == 4 ? 2 : env_slots == 2 ? 1 : (sizeof(BT) == 2 ? 2 : 1)};
+    PipeCfg cfg{0, 0, env_slots == 4 ? 2 : env_slots == 2 ? 1 : (sizeof(BT) == 2 ? 2 : 1), -1};
+#if DELTALOG_TEST_HOOKS
+    cfg.test_drop_item = env_int_now("DELTALOG_TEST_DROP_ITEM", -1);
+#endif
     int ctas = env_ctas > 0 ? env_ctas : 1;
     if (pipelined) {
         const int aux = AuxLayout<OP, D, IO, UL>(st.cap).bytes;
@@ -241,13 +200,17 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
             // aux stages: two are held by the scalar group (unit i and i+1), the rest is prefetch
             for (cfg.n_aux = want_aux; cfg.n_aux >= 2; --cfg.n_aux) {
                 cfg.n_base = (budget - fixed - cfg.n_aux * aux) / kStage;
-                if (cfg.n_base >= want_base || (cfg.n_aux == 2 && cfg.n_base >= 2)) break;
+                if (cfg.n_base >= want_base || cfg.n_aux == 2) break;
             }
-            if (cfg.n_aux >= 2) break;
+            // Each chunk of a tile has its own producer warp, which refills a stage as soon as THAT chunk has
+            // been consumed; a warp's successive chunks are kChunks apart in the ring, so with fewer than
+            // kChunks stages it would wait for a phase of the stage's barrier that it cannot tell from the
+            // one before (one-bit parity).  The ring must hold at least one whole tile.
+            if (cfg.n_base >= kChunks) break;
         }
-        if (ctas < 1) pipelined = false;
+        if (ctas < 1) pipelined = false;  // the aux stages leave no room for a tile: one CTA per unit instead
         if (cfg.n_base > 8 * (kChunkBytes / kStage)) cfg.n_base = 8 * (kChunkBytes / kStage);
-        if (env_base > 0 && cfg.n_base > env_base) cfg.n_base = env_base;
+        if (env_base > 0 && cfg.n_base > env_base) cfg.n_base = env_base > kChunks ? env_base : kChunks;
     }
     if (pipelined) {
         // What L2 holds on to across steps is about half its size on this part (measured: a re-read set is
@@ -499,11 +462,15 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
                               const void *host_k, const void *host_v, const float *host_g,
                               const float *host_beta, const float *u_bonus,
                               const int32_t *slot_idx, int32_t B, void *host_out, void *stream) {
+    // every check of the decode step runs before the first copy is enqueued: a rejected call leaves the
+    // stream and the staging buffers as they were
     if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
     if (!staging || !host_q || !host_k || !host_v || !host_out) return DELTALOG_ERR_INVALID_ARG;
     if (op_has_gate(desc->op) && (!host_g || !staging->g)) return DELTALOG_ERR_INVALID_ARG;
     if (op_delta_rule(desc->op) && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
-    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
+    if (int rc = validate_token(desc, staging->q, staging->k, staging->v, staging->g, staging->beta, u_bonus, B, staging->out))
+        return rc;
     if (B == 0) return DELTALOG_OK;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t units = (size_t)B * desc->H;
@@ -511,7 +478,6 @@ int deltalog_decode_step_host(const deltalog_desc *desc, const deltalog_state *s
     const size_t vec = units * desc->d_v * esz;
     const size_t qk_vec = (size_t)B * qk_heads(desc) * desc->d_k * esz;
     const size_t gbytes = units * (op_vec_decay(desc->op) ? desc->d_k : 1) * sizeof(float);
-    if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
     bool ok = true;
     if (const size_t block = packed_block_bytes(desc, staging, host_q, host_k, host_v, host_g, host_beta, qk_vec, vec,
                                                 gbytes, units)) {
@@ -541,12 +507,13 @@ int deltalog_decode_step_host_overlapped(const deltalog_desc *desc, const deltal
                                          const float *host_g, const float *host_beta, const float *u_bonus,
                                          const int32_t *slot_idx, int32_t B, void *host_out) {
     if (int rc = validate_desc(desc)) return rc;
+    if (int rc = validate_state(state)) return rc;
     if (!staging || !lane || !host_q || !host_k || !host_v || !host_out) return DELTALOG_ERR_INVALID_ARG;
     if (!lane->in_done || !lane->compute_done || !lane->out_done) return DELTALOG_ERR_INVALID_ARG;
     if (op_has_gate(desc->op) && (!host_g || !staging->g)) return DELTALOG_ERR_INVALID_ARG;
     if (op_delta_rule(desc->op) && (!host_beta || !staging->beta)) return DELTALOG_ERR_INVALID_ARG;
-    if (!staging->q || !staging->k || !staging->v || !staging->out) return DELTALOG_ERR_INVALID_ARG;
-    if (B < 0) return DELTALOG_ERR_INVALID_ARG;
+    if (int rc = validate_token(desc, staging->q, staging->k, staging->v, staging->g, staging->beta, u_bonus, B, staging->out))
+        return rc;
     if (B == 0) return DELTALOG_OK;
     cudaStream_t s_in = static_cast<cudaStream_t>(lane->copy_in_stream);
     cudaStream_t s_cmp = static_cast<cudaStream_t>(lane->compute_stream);
@@ -603,7 +570,12 @@ const char *deltalog_status_string(int code) {
     }
 }
 
-int deltalog_version(void) { return 100; }
+int deltalog_version(void) { return 200; }
+
+#ifndef DELTALOG_BUILD_ID
+#define DELTALOG_BUILD_ID "unknown"
+#endif
+const char *deltalog_build_id(void) { return DELTALOG_BUILD_ID; }
 
 uint64_t deltalog_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -8,6 +8,7 @@
 #include <cuda_runtime.h>
 
 #include "deltalog.h"
+#include "validate.h"
 
 namespace {
 
@@ -42,18 +43,28 @@ extern "C" int deltalog_decode_step_host_static(const deltalog_desc *desc, const
                                                 const float *host_g, const float *host_beta,
                                                 const float *u_bonus, const int32_t *slot_idx, int32_t B,
                                                 void *host_out, void *stream) {
+    // Every argument check of the step runs here, before anything touches the shared array or the
+    // stream: a call that is going to be rejected must not clobber what an earlier call staged.
     if (!desc || B < 0 || desc->H <= 0 || desc->d_k <= 0 || desc->d_v <= 0) return DELTALOG_ERR_INVALID_ARG;
     if (desc->io_dtype != DELTALOG_F32 && desc->io_dtype != DELTALOG_BF16) return DELTALOG_ERR_INVALID_ARG;
+    if (int rc = deltalog::validate_desc(desc)) return rc;
+    if (!host_q || !host_k || !host_v || !host_out) return DELTALOG_ERR_INVALID_ARG;
+    if (deltalog::op_has_gate(desc->op) && !host_g) return DELTALOG_ERR_INVALID_ARG;
+    if (deltalog::op_delta_rule(desc->op) && !host_beta) return DELTALOG_ERR_INVALID_ARG;
+    if (desc->op == DELTALOG_RWKV6 && !u_bonus) return DELTALOG_ERR_INVALID_ARG;
     if (B == 0) return DELTALOG_OK;
 
     // carve q | k | v | g | beta | out out of the static area, 256-byte aligned each
     const size_t units = (size_t)B * (size_t)desc->H;
     const size_t esz = desc->io_dtype == DELTALOG_F32 ? 4 : 2;
-    const size_t qk = round256(units * (size_t)desc->d_k * esz);
+    const size_t qk_heads = desc->H_qk > 0 ? (size_t)desc->H_qk : (size_t)desc->H;  // grouped heads: q, k are [B, H_qk, d_k]
+    const size_t qk = round256((size_t)B * qk_heads * (size_t)desc->d_k * esz);
     const size_t vo = round256(units * (size_t)desc->d_v * esz);
     const size_t gb = round256(units * (size_t)(desc->op == DELTALOG_KDA || desc->op == DELTALOG_RWKV6 || desc->op == DELTALOG_GLA ? desc->d_k : 1) * sizeof(float));
     const size_t bb = round256(units * sizeof(float));
     if (2 * qk + 2 * vo + gb + bb > (size_t)DELTALOG_STATIC_STAGING_BYTES) return DELTALOG_ERR_STATIC_LIMIT;
+
+    if (int rc = deltalog::validate_state(state)) return rc;
 
     void *base = nullptr;
     if (int rc = staging_address(&base)) return rc;
