@@ -382,6 +382,17 @@ class Region:
             self.launches = rig.dl.launch_count() - count0
 
 
+def run_region_once(rig: Rig, steps: int, use_graph: bool) -> Region:
+    """Empty the logs, then run exactly ``steps`` steps the way the timed region runs them (untimed)."""
+    region = Region(rig, steps, use_graph)
+    rig.reset_logs()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(region.stream):
+        region.enqueue()
+    torch.cuda.synchronize()
+    return region
+
+
 def timed_passes(rig: Rig, enqueue, stream, clocks: "ClockSampler | None", device, reset=None):
     """Time the region ``enqueue`` puts on ``stream``: logs emptied, barrier + synchronize, events on the
     launching stream around the region, synchronize + barrier.  The first pass decides how often the
@@ -390,6 +401,7 @@ def timed_passes(rig: Rig, enqueue, stream, clocks: "ClockSampler | None", devic
     milliseconds, each the maximum over ranks."""
     reset = reset or rig.reset_logs
     reset()                       # one untimed pass first: graph upload, instruction caches, clocks
+    torch.cuda.synchronize()      # (the reset runs on another stream than the region)
     with torch.cuda.stream(stream):
         enqueue()
     torch.cuda.synchronize()

@@ -58,13 +58,11 @@ def test_chained_graph_replays_equal_plain_launches():
     def run(chain, use_graph):
         rig = bench.Rig(wl, cap, DEV)
         rig.chain = chain
-        rig.reset_logs()
-        if use_graph:
-            bench.time_graph_loop(rig, 2 * bench.graph_steps(cap))
-        else:
-            for t in range(3 * bench.graph_steps(cap)):     # time_graph_loop replays once to warm up
-                rig.step(t)
+        steps = 2 * bench.graph_steps(cap) + 5               # two replays of the cycle graph and a 5-step tail graph
+        region = bench.run_region_once(rig, steps, use_graph)
+        assert region.launches == steps + steps // cap
         assert all(s == 0 for s in rig.status())
+        assert int(rig.states[0].log_len.min()) == int(rig.states[0].log_len.max()) == 5
         return state_snapshot(rig)
 
     ref = run(False, False)
@@ -85,9 +83,7 @@ def test_full_size_config1_in_the_timed_launch_configuration_against_the_oracle(
     uh = torch.tensor([u[1] for u in units], device=DEV)
     rig.reset_logs()
     S0 = f64(rig.states[0].S_base[ub, uh])
-    g_len = bench.graph_steps(cap)
-    bench.time_graph_loop(rig, steps - g_len)            # one warm-up replay + (steps - g_len) timed = `steps` steps
-    torch.cuda.synchronize()
+    bench.run_region_once(rig, steps, use_graph=True)
     assert all(s == 0 for s in rig.status()) and int(rig.states[0].log_len.abs().sum()) == 0
     ring = rig.rings[0]
     pick = lambda name: np.stack([f64(ring[t % rig.RING][name][ub, uh]).reshape(len(units), -1) for t in range(steps)])
