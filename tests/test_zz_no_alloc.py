@@ -32,6 +32,17 @@ def test_requests_beyond_the_built_in_area_are_rejected_on_the_host():
                                               0x90000, None)
     assert rc == binding.ERR_STATIC_LIMIT
     assert "staging" in dl.status_string(rc)
+    # the limit is sharp: 254 rows fit (checked on the GPU below), 255 do not
+    assert lib.deltalog_decode_step_host_static(ctypes.byref(desc), ctypes.byref(st), *fake, None, None, 255,
+                                                0x90000, None) == binding.ERR_STATIC_LIMIT
+    # grouped heads stage fewer query / key rows: with 8 query/key heads 300 rows fit, so the request is judged
+    # on its other arguments (here: a state pointer that is not 16-byte aligned)
+    grouped = dl.Desc(op=dl.GDN, num_slots=512, H=32, d_k=128, d_v=128, cap=8, H_qk=8).c_struct()
+    bad_state = binding._State(0x1008, *(0x1000 * (i + 2) for i in range(5)))
+    assert lib.deltalog_decode_step_host_static(ctypes.byref(grouped), ctypes.byref(bad_state), *fake, None, None, 300,
+                                                0x90000, None) == binding.ERR_INVALID_ARG
+    assert lib.deltalog_decode_step_host_static(ctypes.byref(desc), ctypes.byref(bad_state), *fake, None, None, 300,
+                                                0x90000, None) == binding.ERR_STATIC_LIMIT
     assert lib.deltalog_decode_step_host_static(ctypes.byref(desc), ctypes.byref(st), *fake, None, None, -1,
                                                 0x90000, None) == binding.ERR_INVALID_ARG
     assert lib.deltalog_decode_step_host_static(None, ctypes.byref(st), *fake, None, None, 1, 0x90000, None) == \
@@ -71,3 +82,29 @@ def test_static_staging_matches_the_caller_staged_entry_point_on_two_calls_in_a_
         assert torch.equal(a, b)
     assert int(new_state.status.item()) == 0
     assert int(new_state.log_len.max()) == 2
+
+
+@pytest.mark.gpu
+def test_a_request_that_fills_the_built_in_area_to_the_last_block():
+    """254 rows of the benchmark shape (bf16, 32 heads, head size 128) use 8 388 096 of the 8 388 608
+    bytes: the output region is the last carve-out and ends 512 bytes below the top of the array."""
+    import paper_2608_15533_b200 as dl
+
+    dev = "cuda"
+    wl = Workload("noalloc_limit", GDN, 254, 32, 128, 2, (4,))
+    src = workloads.TokenSource(wl, device=dev)
+    S0 = src.initial_state()
+    desc = make_desc(wl, 4)
+    ref_state, new_state = dl.State(desc, S0.clone()), dl.State(desc, S0.clone())
+    staging = dl.HostStaging(desc, wl.batch, dev)
+    for call in range(2):
+        tok = {k: (v.cpu().pin_memory() if v is not None else None) for k, v in src.token().items()}
+        out_ref = torch.zeros(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()
+        out_new = torch.ones(wl.batch, wl.H, wl.d, dtype=wl.io_dtype).pin_memory()
+        dl.decode_step_host(desc, ref_state, staging, tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], out_ref)
+        dl.decode_step_host_static(desc, new_state, tok["q"], tok["k"], tok["v"], tok["g"], tok["beta"], out_new)
+        torch.cuda.synchronize()
+        assert torch.equal(out_new, out_ref), f"call {call}"
+        assert bool(out_new[-1].float().abs().sum() > 0)            # the last row, at the top of the array, was produced
+    assert torch.equal(ref_state.U_log, new_state.U_log) and torch.equal(ref_state.log_len, new_state.log_len)
+    assert int(new_state.status.item()) == 0 and int(new_state.log_len.min()) == 2
