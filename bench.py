@@ -591,6 +591,90 @@ def time_paper_cycle(rig: Rig, steps: int):
     return steps, total, fused_ms
 
 
+class PhaseGraphs:
+    """The paper's cycle the way a runtime that replays ONE graph per decode step runs it (Section 4):
+    two phase-specialised CUDA graphs per batch descriptor -- an append graph holding one
+    ``deltalog_decode_step`` and a merge graph holding one ``deltalog_decode_merge_step`` -- captured once
+    over FIXED token, slot-list and output buffers; every step the host (which knows each row's phase
+    from its step counter) refreshes the buffers and replays the graph of the phase.
+
+    Uniform batch: all rows are in the same phase, one replay per step.  Staggered batch: both graphs are
+    replayed every step over phase-split slot lists (a row sits out of a call with slot -1).  The token of
+    a step reaches the fixed buffers with one device copy from the packed token ring, standing in for
+    the projections that would write there."""
+
+    def __init__(self, rig: Rig, layer: int = 0):
+        dl = rig.dl
+        self.rig, self.layer = rig, layer
+        self.names = [k for k, v in rig.rings[layer][0].items() if v is not None]
+        # token ring and the fixed buffers in one packed layout (256-byte aligned sections): one copy per step
+        spans, off = {}, 0
+        for k in self.names:
+            t = rig.rings[layer][0][k]
+            spans[k] = (off, t.numel() * t.element_size(), t.dtype, t.shape)
+            off += (t.numel() * t.element_size() + 255) // 256 * 256
+        self.packed_ring = []
+        for tok in rig.rings[layer]:
+            block = torch.zeros(off, dtype=torch.uint8, device=rig.device)
+            for k in self.names:
+                o, nb, _, _ = spans[k]
+                block[o:o + nb].copy_(tok[k].reshape(-1).view(torch.uint8))
+            self.packed_ring.append(block)
+        self.fixed = torch.zeros(off, dtype=torch.uint8, device=rig.device)
+        self.tok = {k: self.fixed[o:o + nb].view(dt).view(shape) for k, (o, nb, dt, shape) in spans.items()}
+        B = rig.wl.batch
+        rows = rig.slot_idx if rig.slot_idx is not None else torch.arange(B, dtype=torch.int32, device=rig.device)
+        self.rows = rows
+        self.app_slots, self.mrg_slots = rows.clone(), rows.clone()
+        self.stream = torch.cuda.Stream(device=rig.device)
+        args = (rig.desc, rig.states[layer], self.tok["q"], self.tok["k"], self.tok["v"], self.tok.get("g"))
+        kw = dict(beta=self.tok.get("beta"), u_bonus=rig.bonus[layer], out=rig.out)
+        for fn, slots in ((dl.decode_step, self.app_slots), (dl.decode_merge_step, self.mrg_slots)):
+            fn(*args, slot_idx=torch.full_like(rows, -1), **kw)     # first launch of the kernel outside any capture
+        torch.cuda.synchronize()
+        self.append_graph, self.merge_graph = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.stream(self.stream):
+            with torch.cuda.graph(self.append_graph, stream=self.stream):
+                dl.decode_step(*args, slot_idx=self.app_slots, **kw)
+            with torch.cuda.graph(self.merge_graph, stream=self.stream):
+                dl.decode_merge_step(*args, slot_idx=self.mrg_slots, **kw)
+        torch.cuda.synchronize()
+
+    def step(self, t: int, merge_rows=None):
+        """Step ``t`` on ``self.stream``.  Uniform batch: ``merge_rows`` is None and the phase follows from
+        ``t`` (every (cap + 1)-th step is the merge step).  Staggered batch: ``merge_rows`` is the boolean
+        mask of the rows whose log is full."""
+        self.fixed.copy_(self.packed_ring[t % self.rig.RING], non_blocking=True)
+        if merge_rows is None:
+            (self.merge_graph if t % (self.rig.cap + 1) == self.rig.cap else self.append_graph).replay()
+            return
+        skip = torch.full_like(self.rows, -1)
+        self.app_slots.copy_(torch.where(merge_rows, skip, self.rows))
+        self.mrg_slots.copy_(torch.where(merge_rows, self.rows, skip))
+        self.append_graph.replay()
+        self.merge_graph.replay()
+
+
+def time_phase_graphs(rig: Rig, steps: int):
+    """The paper's cycle on a uniform single-layer batch through ``PhaseGraphs``: one graph replay per step,
+    selected by the host's step counter.  Returns (steps timed, total ms)."""
+    M = rig.cap + 1
+    steps = max(steps // M, 2) * M
+    rig.reset_logs()
+    pg = PhaseGraphs(rig)
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(pg.stream):
+        for t in range(M):          # one untimed cycle
+            pg.step(t)
+        start.record()
+        for t in range(steps):
+            pg.step(t)
+        end.record()
+    torch.cuda.synchronize()
+    return steps, start.elapsed_time(end)
+
+
 def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = True):
     """The eager dense comparator on the same token ring, launched the same way as the main loop (a
     graph of one trip round the token ring, replayed; the step count is rounded to whole trips, at
@@ -1003,6 +1087,11 @@ def main():
             fused_bytes = (traffic.fused_read(u, cap) + traffic.fused_write(u)) * units
             line["paper_cycle"]["fused_step_ms"] = fused_ms
             line["paper_cycle"]["fused_step_algorithmic_gbs"] = fused_bytes / (fused_ms * 1e-3) / 1e9
+        if not stag and layers == 1:   # the same cycle as two phase-specialised graphs, one replay per step
+            g_steps, g_ms = time_phase_graphs(rig, K)
+            line["paper_cycle"]["phase_graphs"] = {
+                "ms_per_step": g_ms / g_steps, "steps": g_steps,
+                "launch": "an append graph and a merge graph over fixed buffers; per step one token copy and one replay, chosen by the host's step counter"}
         rig.check_status("paper cycle")
         # capacity sweep: whole cycles (at least 32 steps' worth), write reduction per capacity
         sweep = {}

@@ -3,9 +3,10 @@
 sweep with the U-shaped latency curve, state-size scaling, the split-preparation ablation and the
 per-phase costs).  Synthetic inputs of configuration 1's shape (GDN, H = 32, d = 128, bf16 I/O).
 
-    python bench_studies.py [--study m_sweep|state_size|phases|ablation|precision|multi_token|all] [--steps K]
+    python bench_studies.py [--study m_sweep|state_size|phases|ablation|precision|multi_token|all] [--steps K] [--small]
 
-Prints one JSON object per study.  Everything is timed with CUDA events on the launch stream after
+Prints one JSON object per study.  ``--small`` runs every study on a few rows and points (seconds in all):
+it exists so that a test can check that each study runs and what it prints.  Everything is timed with CUDA events on the launch stream after
 warm-up; cycles are replayed from CUDA graphs exactly as in bench.py, whose rig this script reuses.
 One GPU, no CPU path.
 """
@@ -27,6 +28,20 @@ from paper_2608_15533_b200 import traffic
 
 CAPS = (1, 2, 3, 4, 6, 8, 12, 16, 24, 32, 48, 64)
 BATCHES = (4, 8, 16, 32, 64, 128, 256, 512)
+SMALL = False   # --small: a few rows, a few points
+
+
+def base_workload():
+    wl = workloads.CONFIGS[1]
+    return wl.scaled(batch=8, name="gdn_b8_h32_d128") if SMALL else wl
+
+
+def caps():
+    return (1, 3, 4, 16) if SMALL else CAPS
+
+
+def batches():
+    return (2, 8) if SMALL else BATCHES
 
 
 def _steps_for(g_len: int, steps: int) -> int:
@@ -39,16 +54,22 @@ def _split_cycle_ms(rig: bench.Rig, steps: int) -> float:
         rig.step(t)
     rig.reset_logs()
     n = _steps_for(bench.graph_steps(rig.cap), steps)
-    return bench.time_graph_loop(rig, n) / n
+    region = bench.Region(rig, n, use_graph=True)
+    return statistics.median(bench.timed_passes(rig, region.enqueue, region.stream, None, rig.device)) / n
+
+
+def _eager_ms(rig: bench.Rig, steps: int) -> float:
+    n, total = bench.time_eager_loop(rig, rig.states[0].S_base, steps)
+    return total / n
 
 
 def study_m_sweep(device, steps: int) -> dict:
     """Latency against the log capacity: both cycles, with the byte model beside the measurement."""
-    wl = workloads.CONFIGS[1]
+    wl = base_workload()
     u = bench.unit_shape(wl)
     eager_bytes = traffic.eager_read(u) + traffic.eager_write(u)
     rows = []
-    for cap in CAPS:
+    for cap in caps():
         rig = bench.Rig(wl, cap, device)
         split_ms = _split_cycle_ms(rig, steps)
         p_steps, p_ms, fused_ms = bench.time_paper_cycle(rig, steps)
@@ -66,7 +87,7 @@ def study_m_sweep(device, steps: int) -> dict:
         del rig
         torch.cuda.empty_cache()
     rig = bench.Rig(wl, 16, device)
-    eager_ms = bench.time_eager_loop(rig, rig.states[0].S_base, _steps_for(rig.RING, steps)) / _steps_for(rig.RING, steps)
+    eager_ms = _eager_ms(rig, steps)
     best = min(rows, key=lambda r: r["split_us_per_step"])
     return {"study": "m_sweep", "workload": wl.name, "eager_us_per_step": eager_ms * 1e3,
             "eager_bytes_per_unit_step": eager_bytes, "best_cap_split": best["cap"], "rows": rows}
@@ -78,14 +99,13 @@ def study_state_size(device, steps: int) -> dict:
     base = workloads.CONFIGS[1]
     u = bench.unit_shape(base)
     rows = []
-    for batch in BATCHES:
+    for batch in batches():
         wl = base.scaled(batch=batch, name=f"gdn_b{batch}_h32_d128")
         rig = bench.Rig(wl, 16, device)
         split_ms = _split_cycle_ms(rig, steps)
         p_steps, p_ms, _ = bench.time_paper_cycle(rig, steps)
         rig.reset_logs()
-        n = _steps_for(rig.RING, steps)
-        eager_ms = bench.time_eager_loop(rig, rig.states[0].S_base, n) / n
+        eager_ms = _eager_ms(rig, steps)
         assert all(s == 0 for s in rig.status())
         cyc = traffic.cycle_bytes(u, 16)
         rows.append({"batch": batch, "state_mib": wl.units * u.state / 2**20,
@@ -101,7 +121,7 @@ def study_phases(device, steps: int) -> dict:
     """Cost of each launch of a cycle at cap 16: the decode step at every log fill (does appending
     get slower as the log grows?), the token-less merge and the fused merge step.  Plain launches with
     one event pair around each; the cost of an empty event pair is reported beside them."""
-    wl, cap = workloads.CONFIGS[1], 16
+    wl, cap = base_workload(), 16
     rig = bench.Rig(wl, cap, device)
     ev = lambda: torch.cuda.Event(enable_timing=True)
     per_fill = [[] for _ in range(cap)]
@@ -145,9 +165,9 @@ def study_ablation(steps: int) -> dict:
                              env=env, capture_output=True, text=True, check=True).stdout.strip().splitlines()[-1]
         line = json.loads(out)
         rows.append({"variant": name, "us_per_step": line["ms_per_step"] * 1e3,
-                     "decode_us": line["amortized"]["decode_ms_per_step"] * 1e3,
+                     "decode_us": line["amortized"]["decode_ms_per_launch"] * 1e3,
                      "plain_launch_us_per_step": line["amortized"]["plain_launch_ms_per_step"] * 1e3,
-                     "decode_frac_of_measured_peak": line["roofline"]["frac"]})
+                     "decode_algorithmic_frac_of_measured_peak": line["roofline"]["frac_algorithmic_incl_l2"]})
     return {"study": "ablation", "workload": workloads.CONFIGS[1].name, "cap": 16, "rows": rows}
 
 
@@ -157,10 +177,10 @@ def study_precision(device, steps: int) -> dict:
     16-bit dense state (tests/test_gpu_bf16_base.py): half the dense bytes, for the log schedule and for
     the eager kernel, per capacity -- with a smaller base the replay of the log weighs more, so the best
     capacity moves down."""
-    wl = workloads.CONFIGS[1]
+    wl = base_workload()
     rows = []
     variants = [("fp32 state, U log fp32 (default)", False, False, 16), ("fp32 state, U log bf16", True, False, 16)]
-    variants += [(f"bf16 state, U log fp32, cap {c}", False, True, c) for c in (4, 8, 16, 32)]
+    variants += [(f"bf16 state, U log fp32, cap {c}", False, True, c) for c in ((8,) if SMALL else (4, 8, 16, 32))]
     variants += [("bf16 state, U log bf16, cap 16", True, True, 16)]
     for name, u16, b16, cap in variants:
         rig = bench.Rig(wl, cap, device, ulog16=u16, base16=b16)
@@ -173,7 +193,7 @@ def study_precision(device, steps: int) -> dict:
                "write_reduction_vs_eager": cyc["write_reduction"]}
         if cap == 16 and not u16:
             rig.reset_logs()
-            e_ms = bench.time_eager_loop(rig, rig.states[0].S_base, _steps_for(rig.RING, steps)) / _steps_for(rig.RING, steps)
+            e_ms = _eager_ms(rig, steps)
             row["eager_us_per_step"] = e_ms * 1e3
             row["eager_hbm_gbs"] = (traffic.eager_read(u) + traffic.eager_write(u)) * wl.units / (e_ms * 1e-3) / 1e9
             row["speedup_vs_eager_kernel"] = e_ms / ms
@@ -189,11 +209,11 @@ def study_multi_token(device, steps: int) -> dict:
     merge, replayed from a CUDA graph.  Per-token cost and algorithmic bytes."""
     import paper_2608_15533_b200 as dl
 
-    wl, cap = workloads.CONFIGS[1], 16
+    wl, cap = base_workload(), 16
     rig = bench.Rig(wl, cap, device)
     u = bench.unit_shape(wl)
     rows = []
-    for T in (1, 2, 4, 8, 16):
+    for T in ((1, 4) if SMALL else (1, 2, 4, 8, 16)):
         blocks = [{k: (torch.stack([rig.rings[0][(i * T + t) % rig.RING][k] for t in range(T)], dim=1).contiguous()
                        if rig.rings[0][0][k] is not None else None) for k in rig.rings[0][0]}
                   for i in range(rig.RING)]
@@ -245,7 +265,10 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--study", default="all", choices=["m_sweep", "state_size", "phases", "ablation", "precision", "multi_token", "all"])
     ap.add_argument("--steps", type=int, default=1024)
+    ap.add_argument("--small", action="store_true", help="a few rows and a few points per study (a smoke run)")
     args = ap.parse_args()
+    global SMALL
+    SMALL = args.small
     assert torch.cuda.is_available(), "the studies need a CUDA device (there is no CPU path)"
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)

@@ -92,3 +92,50 @@ def test_full_size_config1_in_the_timed_launch_configuration_against_the_oracle(
     assert err <= TOL_STATE, f"state error {err:.3e}"
     out_err = rel_err(f64(rig.out[ub, uh]), ref["out"][-1])
     assert out_err <= 2e-2, f"output error {out_err:.3e}"
+
+
+@pytest.mark.parametrize("staggered", [False, True])
+def test_two_phase_specialised_graphs_equal_the_sequential_paper_cycle(staggered):
+    """An append graph and a merge graph over fixed buffers, selected (uniform batch) or both replayed over
+    phase-split slot lists (staggered fills) by the host, against plain calls of the same cycle:
+    bit-identical state, log and outputs at every step."""
+    import paper_2608_15533_b200 as dl
+
+    wl = Workload("phase_graphs", GDN, 48, 4, 128, 40, (4,), num_slots=64 if staggered else None, staggered=staggered)
+    cap, M, steps = 4, 5, 23
+
+    def fills(rig):   # staggered: row b starts `delay` steps late, so the rows' logs fill at different steps
+        return workloads.fill_offsets(wl, M).to(DEV) if staggered else torch.zeros(wl.batch, dtype=torch.long, device=DEV)
+
+    def run(use_graphs):
+        rig = bench.Rig(wl, cap, DEV)
+        delay = fills(rig)
+        rows = rig.slot_idx if rig.slot_idx is not None else torch.arange(wl.batch, dtype=torch.int32, device=DEV)
+        skip = torch.full_like(rows, -1)
+        pg = bench.PhaseGraphs(rig) if use_graphs else None
+        outs = []
+        stream = pg.stream if pg else torch.cuda.current_stream()
+        with torch.cuda.stream(stream):
+            for t in range(steps):
+                age = t - delay                                  # steps a row has taken part in
+                active = age >= 0
+                full = active & (age % M == cap)                 # its log holds cap entries: merge phase
+                tok = rig.rings[0][t % rig.RING]
+                if use_graphs:
+                    if staggered:
+                        pg.rows = torch.where(active, rows, skip)
+                        pg.step(t, merge_rows=full)
+                    else:
+                        pg.step(t)
+                else:
+                    args = (rig.desc, rig.states[0], tok["q"], tok["k"], tok["v"], tok["g"])
+                    dl.decode_step(*args, beta=tok["beta"], slot_idx=torch.where(active & ~full, rows, skip), out=rig.out)
+                    dl.decode_merge_step(*args, beta=tok["beta"], slot_idx=torch.where(full, rows, skip), out=rig.out)
+                outs.append(rig.out.clone())
+        torch.cuda.synchronize()
+        assert all(s == 0 for s in rig.status())
+        return state_snapshot(rig), torch.stack(outs)
+
+    (ref, out_ref), (got, out_got) = run(False), run(True)
+    assert same(ref, got) and torch.equal(out_ref, out_got)
+    assert int(ref[0][4].max()) > 0                                  # logs are in use at the end
