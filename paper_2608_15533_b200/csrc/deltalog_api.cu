@@ -12,6 +12,7 @@
 #include "decode_kernel.cuh"
 #include "decode_multi_kernel.cuh"
 #include "decode_pipelined.cuh"
+#include "decode_pipelined_d64.cuh"
 #include "eager_kernel.cuh"
 #include "fused_step_kernel.cuh"
 #include "merge_kernel.cuh"
@@ -174,7 +175,7 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
     // every unit's snapshot row to start on a 16-byte boundary: cap % 4 == 0 for GDN.
     // Head size 64: a unit is a single 16 KiB chunk and the per-unit hand-overs of the pipeline cost
     // more than they hide, so the one-CTA-per-unit kernel is the faster one there (measured).
-    bool pipelined = impl != 1 && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0) && (D == 128 || impl == 2);
+    bool pipelined = impl != 1 && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0) && (D == 128 || (impl == 2 && sizeof(BT) == 2));
     constexpr int kStage = chunk_bytes<D, BT>();
     constexpr int kChunks = D * D * (int)sizeof(BT) / kStage;  // chunks per base tile
     // hand-over slots: two while the base tile's arrival sets the pace; with a 16-bit base the chain
@@ -229,6 +230,26 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
         if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, grid, kPipeThreads, smem, stream, st, tk, cfg);
         kernel<<<grid, kPipeThreads, smem, stream>>>(st, tk, cfg);
         return finish_launch();
+    }
+    if constexpr (D == kP64D && std::is_same<BT, float>::value) {
+        // Head size 64, fp32 base: the persistent kernel with warp-per-unit roles, whose aux stages are sized by
+        // the live log length inside the kernel.  It needs room for at least four stages at the full capacity
+        // beside the 8-tile base ring (always true up to capacity 32 or so), and 16-byte aligned snapshot rows.
+        static const int env_aux_kb = env_int("DELTALOG_P64_AUX_KB", 0);
+        P64Cfg c64{8, 8, 0};
+        const int budget = (dev.smem_optin < dev.smem_per_sm - 1024 ? dev.smem_optin : dev.smem_per_sm - 1024);
+        c64.aux_bytes = (budget - p64_smem_bytes(c64)) / 128 * 128;
+        if (env_aux_kb > 0 && env_aux_kb * 1024 < c64.aux_bytes) c64.aux_bytes = env_aux_kb * 1024;
+        const bool fits = c64.aux_bytes >= 4 * AuxLayout<OP, D, IO, UL>(st.cap).bytes;
+        if (impl != 1 && dev.sms > 0 && fits && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
+            auto kernel = decode_pipelined_d64_kernel<OP, IO, UL>;
+            const int smem = p64_smem_bytes(c64);
+            if (int rc = ensure_smem(kernel, smem)) return rc;
+            const int grid = total < dev.sms ? total : dev.sms;
+            if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, grid, kP64Threads, smem, stream, st, tk, c64);
+            kernel<<<grid, kP64Threads, smem, stream>>>(st, tk, c64);
+            return finish_launch();
+        }
     }
     auto kernel = decode_append_kernel<OP, D, IO, UL, BT>;
     const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
