@@ -17,13 +17,17 @@
 //   epilogue warps (4 warps)  warp e owns units e, e+4, ...: value-side replay, b, the output and the
 //                             append.
 //
-// How many units an SM keeps in flight is set by the aux ring: a unit holds its stage from the moment
-// its copies are queued until its epilogue is done (about 5 us), so the ring's depth divided by that
-// time is the unit rate.  A stage sized for the full capacity allows 8 stages beside the 8-tile base
-// ring, which is what the one-CTA-per-unit kernel reaches as well.  The stages are therefore sized by
-// the longest LIVE log among the CTA's units, found in a short prologue (the base producers do not wait
-// for it: the base ring has a fixed place): with a half-full log twice as many stages fit and the
-// kernel runs at the rate of the tile stream.
+// How many units an SM keeps in flight is set by the rings that hold a unit's small operands: a stage
+// is occupied from the moment its copies are queued until its last reader is done, so a ring's depth
+// divided by that time is the unit rate.  Two measures keep that rate above the rate of the tile
+// stream.  (1) The operands travel in two rings with different life times: the key side (K, Lambda,
+// q, k, gate, bonus -- three quarters of the bytes for per-key decay) is read by the prep warp only
+// and released about 3 us after its copies were queued; the value side (U, v) waits for the stream
+// and epilogue warps, about 5 us.  (2) The stages are sized by the longest LIVE log among the CTA's
+// units, found in a short prologue (the base producers do not wait for it: the base ring has a fixed
+// place), and the two depths are chosen for that size.  With one ring of stages sized for the full
+// capacity only 8 units were in flight beside the 8-tile base ring -- the rate of the
+// one-CTA-per-unit kernel.
 //
 // Ring depths are multiples of the number of warps that take turns waiting on a ring, so that a stage
 // is always awaited by the same warp in program order (the one-bit phase parity of an mbarrier wait
@@ -39,10 +43,11 @@ constexpr int kP64D = 64;
 constexpr int kP64StreamWarps = 4;
 constexpr int kP64AuxWarps = 4;
 constexpr int kP64BaseWarps = 2;
-constexpr int kP64MaxAux = 24;             // upper bound on the aux ring's depth (mbarrier storage)
+constexpr int kP64MaxKey = 16;             // upper bounds on the depths of the key-side and value-side rings
+constexpr int kP64MaxVal = 32;             // (mbarrier storage)
 constexpr int kP64Threads = 32 * (kP64StreamWarps + 4 + 4 + kP64BaseWarps + kP64AuxWarps);  // stream, prep, epilogue, base and aux producers
 constexpr int kP64ScalarWarps = 4;         // prep warps, and as many epilogue warps
-constexpr int kP64BarrierBytes = 1024;
+constexpr int kP64BarrierBytes = 2048;
 // hand-over slot (floats): q, k, mul_k, mul_q, lbar, lbar' [6 x 64], ck, cq [2 x 64], scalars [4],
 // the two base-pass results [2][64]
 constexpr int kP64SlotFloats = 6 * 64 + 2 * kMaxCap + 4 + 2 * 64;
@@ -61,10 +66,38 @@ __device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&out)[8]) {
     out[6] = __uint_as_float(v.w << 16), out[7] = __uint_as_float(v.w & 0xffff0000u);
 }
 
+// Byte offsets inside a key-side stage and a value-side stage with room for n log entries.
+template <int OP, typename IO>
+struct KeyStage {
+    static constexpr bool kVec = OpTraits<OP>::kVecDecay;
+    static constexpr int DL = kVec ? kP64D : 1;
+    int K, L, q, k, g, bonus, meta, bytes;
+    __host__ __device__ explicit KeyStage(int n) {
+        K = 0;
+        L = K + n * kP64D * (int)sizeof(IO);
+        q = L + align_up(n * DL * 4, 16);
+        k = q + kP64D * (int)sizeof(IO);
+        g = k + kP64D * (int)sizeof(IO);
+        bonus = g + (kVec ? kP64D * 4 : 0);
+        meta = bonus + (OP == DELTALOG_RWKV6 ? kP64D * 4 : 0);
+        bytes = align_up(meta + 32, 128);
+    }
+};
+template <typename IO, typename UL>
+struct ValStage {
+    int U, v, meta, bytes;
+    __host__ __device__ explicit ValStage(int n) {
+        U = 0;
+        v = U + n * kP64D * (int)sizeof(UL);
+        meta = v + kP64D * (int)sizeof(IO);
+        bytes = align_up(meta + 32, 128);
+    }
+};
+
 struct P64Cfg {
     int n_base;     // stages of the base ring (one 16 KiB tile each), a multiple of 4
     int n_slots;    // hand-over slots, a multiple of 4
-    int aux_bytes;  // bytes of the aux ring's region; its depth follows from the live log lengths
+    int aux_bytes;  // bytes shared by the key-side and value-side rings; their depths follow from the live log lengths
 };
 
 __host__ inline int p64_smem_bytes(P64Cfg cfg) {
@@ -92,8 +125,9 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
     unsigned char *aux_ring = base_ring + (size_t)NB * kChunkBytes;
 
     const uint32_t full_base = smem_addr(bars), empty_base = full_base + 8u * NB;
-    const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * kP64MaxAux;
-    const uint32_t prep_done = empty_aux + 8u * kP64MaxAux;  // [NS] prep warp -> stream warp
+    const uint32_t full_key = empty_base + 8u * NB, empty_key = full_key + 8u * kP64MaxKey;
+    const uint32_t full_val = empty_key + 8u * kP64MaxKey, empty_val = full_val + 8u * kP64MaxVal;
+    const uint32_t prep_done = empty_val + 8u * kP64MaxVal;  // [NS] prep warp -> stream warp
     const uint32_t stream_done = prep_done + 8u * NS;   // [NS] stream warp -> epilogue warp
     const uint32_t coef_done = stream_done + 8u * NS;   // [NS] prep warp -> epilogue warp
     const uint32_t slot_free = coef_done + 8u * NS;     // [NS] epilogue warp -> prep warp
@@ -104,9 +138,13 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
             mbar_init(full_base + 8u * i, 1);
             mbar_init(empty_base + 8u * i, 1);  // the unit's stream warp
         }
-        for (int i = 0; i < kP64MaxAux; ++i) {
-            mbar_init(full_aux + 8u * i, 1);
-            mbar_init(empty_aux + 8u * i, 2);  // the unit's prep warp and its epilogue warp
+        for (int i = 0; i < kP64MaxKey; ++i) {
+            mbar_init(full_key + 8u * i, 1);
+            mbar_init(empty_key + 8u * i, 1);  // the unit's prep warp
+        }
+        for (int i = 0; i < kP64MaxVal; ++i) {
+            mbar_init(full_val + 8u * i, 1);
+            mbar_init(empty_val + 8u * i, 1);  // the unit's epilogue warp
         }
         for (int i = 0; i < NS; ++i) {
             mbar_init(prep_done + 8u * i, 1);
@@ -136,7 +174,7 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
     // Lengths are written by the step before this one, so this is also where a kernel that was started
     // ahead of the preceding kernel's completion waits for it.  The aux producers look the lengths up (one
     // unit per lane), the maximum is combined in shared memory, and the aux ring is laid out for it.
-    int NA = 4;
+    int NK = 4, NV = 4;  // depths of the key-side and the value-side ring
     int stage_cap = 1;   // entries a stage has room for
     if (!is_base_producer) {
         asm volatile("griddepcontrol.wait;\n" ::: "memory");
@@ -159,10 +197,23 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
         stage_cap = max(*max_len_s, 1);
         if (!kVecDecay) stage_cap = align_up(stage_cap, 4);  // scalar snapshots travel in 16-byte pieces
         if (stage_cap > cap) stage_cap = cap;
-        const int fit = cfg.aux_bytes / AuxLayout<OP, D, IO, UL>(stage_cap).bytes;
-        NA = min(kP64MaxAux, fit) & ~3;
+        // Depths (multiples of 4): a key-side stage is occupied for about 3 us (its copies' latency and the
+        // prep warp), a value-side stage for about 5 us, so the unit rate is min(NK / 3, NV / 5) per
+        // microsecond -- take the split that maximises it.  (Measured at 15 live entries of configuration 3:
+        // depths 4 / 20 run at 101 us per launch, 8 / 8 at 75.)
+        const int kb = KeyStage<OP, IO>(stage_cap).bytes, vb = ValStage<IO, UL>(stage_cap).bytes;
+        int best = 0;
+        for (int nk = 4; nk <= kP64MaxKey; nk += 4) {
+            const int nv = min(kP64MaxVal, (cfg.aux_bytes - nk * kb) / vb) & ~3;
+            if (nv < 4) break;
+            const int rate = min(5 * nk, 3 * nv);
+            if (rate > best) best = rate, NK = nk, NV = nv;
+        }
     }
-    const AuxLayout<OP, D, IO, UL> lay(stage_cap);
+    const KeyStage<OP, IO> klay(stage_cap);
+    const ValStage<IO, UL> vlay(stage_cap);
+    unsigned char *key_ring = aux_ring;
+    unsigned char *val_ring = aux_ring + (size_t)NK * klay.bytes;
 
     if (warp >= kP64StreamWarps + 2 * kP64ScalarWarps && warp < kP64StreamWarps + 2 * kP64ScalarWarps + kP64BaseWarps) {
         // ================= base producers: warp b owns units b, b + kP64BaseWarps, ... ==============
@@ -253,47 +304,53 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
                 const float btj = __shfl_sync(0xffffffffu, bt, j);
                 if (lane != 0 || dead) continue;
                 const int i = a + kP64AuxWarps * (n0 + j);
-                const int astg = i % NA;
-                if (!bounded_wait(empty_aux + 8u * astg, ((uint32_t)(i / NA) & 1u) ^ 1u, abort_flag)) {
+                const int ks = i % NK, vs = i % NV;
+                if (!bounded_wait(empty_key + 8u * ks, ((uint32_t)(i / NK) & 1u) ^ 1u, abort_flag) ||
+                    !bounded_wait(empty_val + 8u * vs, ((uint32_t)(i / NV) & 1u) ^ 1u, abort_flag)) {
                     dead = true;
                     continue;
                 }
-                unsigned char *stage = aux_ring + (size_t)astg * lay.bytes;
-                const uint32_t fa = full_aux + 8u * astg;
-                *reinterpret_cast<int4 *>(stage + lay.meta) = make_int4(L, fl, __float_as_int(gsj), __float_as_int(btj));
-                *reinterpret_cast<int *>(stage + lay.meta + 16) = s;
+                unsigned char *kst = key_ring + (size_t)ks * klay.bytes, *vst = val_ring + (size_t)vs * vlay.bytes;
+                const uint32_t fk = full_key + 8u * ks, fv = full_val + 8u * vs;
+                const int4 meta = make_int4(L, fl, __float_as_int(gsj), __float_as_int(btj));
+                *reinterpret_cast<int4 *>(kst + klay.meta) = meta;
+                *reinterpret_cast<int4 *>(vst + vlay.meta) = meta;
+                *reinterpret_cast<int *>(vst + vlay.meta + 16) = s;
                 if (fl != 0) {
-                    mbar_arrive(fa);  // nothing to copy: the compute warps only read the flags
+                    mbar_arrive(fk);  // nothing to copy: the compute warps only read the flags
+                    mbar_arrive(fv);
                 } else {
                     const int item = first + i * stride;
                     const int kb = L * D * (int)sizeof(IO), ub = L * D * (int)sizeof(UL);
                     const int lb = kVecDecay ? L * D * 4 : align_up(L, 4) * 4;
-                    const uint32_t bytes = (L > 0 ? kb + ub + lb : 0) + 3 * io_vec + (kVecDecay ? D * 4 : 0) +
-                                           (OP == DELTALOG_RWKV6 ? D * 4 : 0);
-                    mbar_arrive_expect_tx(fa, bytes);
+                    mbar_arrive_expect_tx(fk, (L > 0 ? kb + lb : 0) + 2 * io_vec + (kVecDecay ? D * 4 : 0) +
+                                                  (OP == DELTALOG_RWKV6 ? D * 4 : 0));
+                    mbar_arrive_expect_tx(fv, (L > 0 ? ub : 0) + io_vec);
                     const size_t unit = (size_t)s * H + item % H;
                     const size_t qk = tk.qk_row(item / H, item % H);
-                    const uint32_t sa = smem_addr(stage);
-                    bulk_copy_g2s(sa + lay.q, static_cast<const IO *>(tk.q) + qk * D, io_vec, fa);
-                    bulk_copy_g2s(sa + lay.k, static_cast<const IO *>(tk.k) + qk * D, io_vec, fa);
-                    if (kVecDecay) bulk_copy_g2s(sa + lay.g, tk.g + (size_t)item * D, D * 4, fa);
+                    const uint32_t ka = smem_addr(kst), va = smem_addr(vst);
+                    bulk_copy_g2s(ka + klay.q, static_cast<const IO *>(tk.q) + qk * D, io_vec, fk);
+                    bulk_copy_g2s(ka + klay.k, static_cast<const IO *>(tk.k) + qk * D, io_vec, fk);
+                    if (kVecDecay) bulk_copy_g2s(ka + klay.g, tk.g + (size_t)item * D, D * 4, fk);
                     if (L > 0) {  // read again by the following steps: kept in L2 as far as it fits
                         const uint64_t keep = l2_policy_keep(st.keep_fraction(L, total, kEntryBytes));
-                        bulk_copy_g2s_hint(sa + lay.L, st.decay_log + unit * cap * DL, lb, fa, keep);
-                        bulk_copy_g2s_hint(sa + lay.K, static_cast<const IO *>(st.K_log) + unit * cap * D, kb, fa, keep);
-                        bulk_copy_g2s_hint(sa + lay.U, static_cast<const UL *>(st.U_log) + unit * cap * D, ub, fa, keep);
+                        bulk_copy_g2s_hint(ka + klay.L, st.decay_log + unit * cap * DL, lb, fk, keep);
+                        bulk_copy_g2s_hint(ka + klay.K, static_cast<const IO *>(st.K_log) + unit * cap * D, kb, fk, keep);
+                        bulk_copy_g2s_hint(va + vlay.U, static_cast<const UL *>(st.U_log) + unit * cap * D, ub, fv, keep);
                     }
-                    bulk_copy_g2s(sa + lay.v, static_cast<const IO *>(tk.v) + (size_t)item * D, io_vec, fa);
-                    if (OP == DELTALOG_RWKV6) bulk_copy_g2s(sa + lay.bonus, tk.u_bonus + (size_t)(item % H) * D, D * 4, fa);
+                    if (OP == DELTALOG_RWKV6) bulk_copy_g2s(ka + klay.bonus, tk.u_bonus + (size_t)(item % H) * D, D * 4, fk);
+                    bulk_copy_g2s(va + vlay.v, static_cast<const IO *>(tk.v) + (size_t)item * D, io_vec, fv);
                 }
                 ++n_done;
             }
         }
         if (dead && lane == 0) {
             if (st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
-            for (int b = 0; b < n_done && kP64AuxWarps * b < NA; ++b) {  // let this warp's copies in flight land
+            for (int b = 0; b < n_done; ++b) {  // let this warp's copies in flight land: its newest units, one per stage
                 const int i = a + kP64AuxWarps * (n_done - 1 - b);
-                bounded_wait(full_aux + 8u * (i % NA), (uint32_t)(i / NA) & 1u, abort_flag + 1);
+                if (kP64AuxWarps * b < NK) bounded_wait(full_key + 8u * (i % NK), (uint32_t)(i / NK) & 1u, abort_flag + 1);
+                if (kP64AuxWarps * b < NV) bounded_wait(full_val + 8u * (i % NV), (uint32_t)(i / NV) & 1u, abort_flag + 1);
+                if (kP64AuxWarps * b >= NV) break;
             }
         }
     } else if (warp < kP64StreamWarps) {
@@ -356,11 +413,12 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
         const int pw = warp - kP64StreamWarps;
         bool alive = true;
         for (int i = pw; i < n_items && alive; i += kP64ScalarWarps) {
-            const int astg = i % NA, sl = i % NS;
-            alive = bounded_wait(full_aux + 8u * astg, (uint32_t)(i / NA) & 1u, abort_flag) &&
+            const int ks = i % NK, sl = i % NS;
+            alive = bounded_wait(full_key + 8u * ks, (uint32_t)(i / NK) & 1u, abort_flag) &&
                     bounded_wait(slot_free + 8u * sl, ((uint32_t)(i / NS) & 1u) ^ 1u, abort_flag);
             if (!alive) break;
-            const unsigned char *stage = aux_ring + (size_t)astg * lay.bytes;
+            const unsigned char *stage = key_ring + (size_t)ks * klay.bytes;
+            const KeyStage<OP, IO> &lay = klay;
             float *slot = slot_of(i);
             const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
             const int len = meta.x, flags = meta.y;
@@ -445,7 +503,7 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(coef_done + 8u * sl);
-                mbar_arrive(empty_aux + 8u * astg);
+                mbar_arrive(empty_key + 8u * ks);   // the key side is not needed any more: its stage is free
             }
         }
         if (!alive && lane == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);
@@ -454,13 +512,14 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
         const int ew = warp - kP64StreamWarps - kP64ScalarWarps;
         bool alive = true;
         for (int i = ew; i < n_items && alive; i += kP64ScalarWarps) {
-            const int astg = i % NA, sl = i % NS;
+            const int vs = i % NV, sl = i % NS;
             const uint32_t par = (uint32_t)(i / NS) & 1u;
             alive = bounded_wait(stream_done + 8u * sl, par, abort_flag) &&
                     bounded_wait(coef_done + 8u * sl, par, abort_flag) &&
-                    bounded_wait(full_aux + 8u * astg, (uint32_t)(i / NA) & 1u, abort_flag);
+                    bounded_wait(full_val + 8u * vs, (uint32_t)(i / NV) & 1u, abort_flag);
             if (!alive) break;
-            const unsigned char *stage = aux_ring + (size_t)astg * lay.bytes;
+            const unsigned char *stage = val_ring + (size_t)vs * vlay.bytes;
+            const ValStage<IO, UL> &lay = vlay;
             const float *slot = slot_of(i);
             const int4 meta = *reinterpret_cast<const int4 *>(stage + lay.meta);
             const int len = meta.x, flags = meta.y;
@@ -468,7 +527,6 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
                 const int slot_id = *reinterpret_cast<const int *>(stage + lay.meta + 16);
                 const int item = first + i * stride;
                 const size_t unit = (size_t)slot_id * H + item % H;
-                const IO *k_a = reinterpret_cast<const IO *>(stage + lay.k);
                 const IO *v_a = reinterpret_cast<const IO *>(stage + lay.v);
                 const UL *U_a = reinterpret_cast<const UL *>(stage + lay.U);
                 const float *red_s = slot + oRED;
@@ -495,7 +553,7 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
                         st_hint(Uout + c, from_f32<UL>(to_f32(v_raw)), keep);  // lossless: U log dtype equals the I/O dtype
                         og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(slot[oSC], to_f32(v_raw), yq));
                     }
-                    st_hint(Kout + c, k_a[c], keep);
+                    st_hint(Kout + c, from_f32<IO>(slot[oK + c]), keep);  // the key as the prep warp widened it: exact
                     if (kVecDecay) st_hint(st.decay_log + (unit * cap + len) * DL + c, slot[oLN + c], keep);
                 }
                 if (lane == 0) {
@@ -506,7 +564,7 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(slot_free + 8u * sl);
-                mbar_arrive(empty_aux + 8u * astg);
+                mbar_arrive(empty_val + 8u * vs);
             }
         }
         if (!alive && lane == 0 && st.status) atomicOr(st.status, DELTALOG_STATUS_TIMEOUT);

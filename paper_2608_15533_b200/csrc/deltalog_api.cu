@@ -232,16 +232,20 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
         return finish_launch();
     }
     if constexpr (D == kP64D && std::is_same<BT, float>::value) {
-        // Head size 64, fp32 base: the persistent kernel with warp-per-unit roles, whose aux stages are sized by
-        // the live log length inside the kernel.  It needs room for at least four stages at the full capacity
+        // Head size 64, fp32 base: the persistent kernel with warp-per-unit roles, whose operand stages are sized by
+        // the live log length inside the kernel.  It needs room for at least four stages of each ring at the full capacity
         // beside the 8-tile base ring (always true up to capacity 32 or so), and 16-byte aligned snapshot rows.
         static const int env_aux_kb = env_int("DELTALOG_P64_AUX_KB", 0);
         P64Cfg c64{8, 8, 0};
         const int budget = (dev.smem_optin < dev.smem_per_sm - 1024 ? dev.smem_optin : dev.smem_per_sm - 1024);
         c64.aux_bytes = (budget - p64_smem_bytes(c64)) / 128 * 128;
         if (env_aux_kb > 0 && env_aux_kb * 1024 < c64.aux_bytes) c64.aux_bytes = env_aux_kb * 1024;
-        const bool fits = c64.aux_bytes >= 4 * AuxLayout<OP, D, IO, UL>(st.cap).bytes;
-        if (impl != 1 && dev.sms > 0 && fits && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
+        const bool fits = c64.aux_bytes >= 4 * (KeyStage<OP, IO>(st.cap).bytes + ValStage<IO, UL>(st.cap).bytes);
+        // Beyond 16 live entries the stages get so large that fewer than eight units are in flight and the
+        // one-CTA-per-unit kernel is the faster one (measured on configuration 3's shape at capacity 32:
+        // 105 - 144 us per launch against ~80 - 95 us from 17 entries on), so it keeps the larger capacities.
+        static const int max_cap = env_int("DELTALOG_P64_MAX_CAP", 16);
+        if (impl != 1 && dev.sms > 0 && fits && st.cap <= max_cap && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
             auto kernel = decode_pipelined_d64_kernel<OP, IO, UL>;
             const int smem = p64_smem_bytes(c64);
             if (int rc = ensure_smem(kernel, smem)) return rc;
