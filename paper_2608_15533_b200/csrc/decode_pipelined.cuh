@@ -97,19 +97,20 @@ template <int D>
 __host__ __device__ constexpr int pipe_scratch_bytes(int slot_shift) {
     return (1 << slot_shift) * align_up(pipe_slot_floats<D>() * 4, 128);
 }
-constexpr int kPipeBarrierBytes = 1024;  // mbarriers (2 x 32 + 2 x 8 + 4 x 4 at most) and the abort flags
+constexpr int kPipeMaxBase = 32;         // upper bounds on the ring depths (mbarrier storage)
+constexpr int kPipeMaxAux = 12;
+constexpr int kPipeBarrierBytes = 1024;  // mbarriers (2 x 32 + 2 x 12 + 4 x 4 at most), the abort flags, the live-length word
 
 struct PipeCfg {
-    int n_base;  // stages of the base ring
-    int n_aux;   // stages of the aux ring
+    int n_base;     // stages of the base ring
+    int aux_bytes;  // bytes of the aux ring's region; its depth follows from the live log lengths (see the kernel)
     int slot_shift;  // log2 of the number of hand-over slots (1 or 2)
     int test_drop_item;  // -1; a unit index only in test builds (DELTALOG_TEST_HOOKS)
 };
 
-template <int OP, int D, typename IO, typename UL, typename BT = float>
-__host__ inline int pipe_smem_bytes(int cap, PipeCfg cfg) {
-    return kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift) + cfg.n_aux * AuxLayout<OP, D, IO, UL>(cap).bytes +
-           cfg.n_base * chunk_bytes<D, BT>();
+template <int D, typename BT = float>
+__host__ inline int pipe_smem_bytes(PipeCfg cfg) {
+    return kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift) + cfg.n_base * chunk_bytes<D, BT>() + cfg.aux_bytes;
 }
 
 // ---- mbarrier / bulk-copy primitives ---------------------------------------------------------
@@ -229,18 +230,18 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     constexpr int SLOT = align_up(pipe_slot_floats<D>() * 4, 128) / 4;  // floats per hand-over slot
 
     extern __shared__ __align__(128) unsigned char smem[];
-    const AuxLayout<OP, D, IO, UL> lay(st.cap);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kPipeBarrierBytes - 16);
+    int *max_len_s = reinterpret_cast<int *>(smem + kPipeBarrierBytes - 32);
     float *scratch = reinterpret_cast<float *>(smem + kPipeBarrierBytes);
-    unsigned char *aux_ring = smem + kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift);
-    unsigned char *base_ring = aux_ring + (size_t)cfg.n_aux * lay.bytes;
+    unsigned char *base_ring = smem + kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift);
+    unsigned char *aux_ring = base_ring + (size_t)cfg.n_base * CHB;
 
-    const int NB = cfg.n_base, NA = cfg.n_aux;
+    const int NB = cfg.n_base;
     const uint32_t full_base = smem_addr(bars), empty_base = full_base + 8u * NB;
-    const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * NA;
+    const uint32_t full_aux = empty_base + 8u * NB, empty_aux = full_aux + 8u * kPipeMaxAux;
     const int SH = cfg.slot_shift, NS = 1 << SH;      // hand-over slots; unit i uses slot i % NS in phase (i / NS) & 1
-    const uint32_t prep_done = empty_aux + 8u * NA;   // [NS] scalar group -> stream group: multipliers ready
+    const uint32_t prep_done = empty_aux + 8u * kPipeMaxAux;   // [NS] scalar group -> stream group: multipliers ready
     const uint32_t stream_done = prep_done + 8u * NS;  // [NS] stream group -> epilogue group: partial sums ready
     const uint32_t coef_done = stream_done + 8u * NS;  // [NS] prep group -> epilogue group: coefficients ready
     const uint32_t slot_free = coef_done + 8u * NS;    // [NS] epilogue group -> prep group: hand-over slot reusable
@@ -251,7 +252,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
             mbar_init(full_base + 8u * i, 1);
             mbar_init(empty_base + 8u * i, kGroupWarps);
         }
-        for (int i = 0; i < NA; ++i) {
+        for (int i = 0; i < kPipeMaxAux; ++i) {
             mbar_init(full_aux + 8u * i, 1);
             mbar_init(empty_aux + 8u * i, kGroupWarps);
         }
@@ -263,6 +264,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;  // separate flag for the drain waits after an abort
+        *max_len_s = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
     }
@@ -276,6 +278,40 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
     const int first = blockIdx.x, stride = gridDim.x;
     const int n_items = (total - first + stride - 1) / stride;
     const int cap = st.cap, H = st.H;
+
+    // ---- the aux ring is laid out for the longest LIVE log among this CTA's units ----------------------
+    // A unit's aux stage holds its live log entries and token vectors from the moment the copies are queued
+    // until its epilogue is done; stages sized for the full capacity leave room for few of them at large
+    // capacities (and used to shrink the base ring).  So the aux producers first look up the lengths of the
+    // CTA's units -- which is also where a kernel started ahead of the preceding kernel's completion waits
+    // for it: the lengths are written by the step before -- and every role but the base producers (the base
+    // ring has a fixed place; its producers start at once) picks the depth up from shared memory.
+    constexpr int kFirstBaseWarp = 2 * kGroupWarps, kFirstAuxWarp = 2 * kGroupWarps + kBaseWarps;
+    const bool is_base_producer = warp >= kFirstBaseWarp && warp < kFirstAuxWarp;
+    int NA = 2, stage_cap = 1;
+    if (!is_base_producer) {
+        if (warp >= kFirstAuxWarp) {
+            asm volatile("griddepcontrol.wait;\n" ::: "memory");
+            int mx = 0;
+            for (int it = (warp - kFirstAuxWarp) * 32 + lane; it < n_items; it += 32 * kAuxWarps) {
+                const int item = first + it * stride;
+                const int slot = tk.slot_idx ? tk.slot_idx[item / H] : item / H;
+                if (slot >= 0 && slot < st.num_slots) {
+                    const int len = st.log_len[(size_t)slot * H + item % H];
+                    if (len > 0 && len < cap) mx = max(mx, len);
+                }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            if (lane == 0 && mx > 0) atomicMax(max_len_s, mx);
+        }
+        asm volatile("bar.sync 3, %0;\n" ::"n"(kPipeThreads - 32 * kBaseWarps) : "memory");
+        stage_cap = max(*max_len_s, 1);
+        if (!kVecDecay) stage_cap = align_up(stage_cap, 4);  // scalar snapshots travel in 16-byte pieces
+        if (stage_cap > cap) stage_cap = cap;
+        NA = min(kPipeMaxAux, cfg.aux_bytes / AuxLayout<OP, D, IO, UL>(stage_cap).bytes);  // >= 2: the launcher's check
+    }
+    const AuxLayout<OP, D, IO, UL> lay(stage_cap);
 
     // hand-over slot fields
     auto slot_ptr = [&](int i) { return scratch + (size_t)(i & (NS - 1)) * SLOT; };
@@ -361,16 +397,9 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
         int n_done = 0;  // own units queued so far
         const int io_vec = D * (int)sizeof(IO);
         // Lengths and log entries are written by the step before this one, and the token tensors
-        // (gate, beta, q, k, v) are typically produced by the launch directly in front of this one: when
-        // this kernel was started ahead of the previous kernel's completion, wait for it before any of
-        // them is read (a no-op otherwise).  Only the slot indices are requested before the wait, and only
-        // when the caller vouched for them.  Everything the other roles do with global memory follows
-        // from what these warps load.
-        bool waited = false;
-        if (!slots_early) {
-            asm volatile("griddepcontrol.wait;\n" ::: "memory");
-            waited = true;
-        }
+        // (gate, beta, q, k, v) are typically produced by the launch directly in front of this one: these
+        // warps have waited for the preceding kernel (in the prologue above) before any of them is read.
+        // Everything the other roles do with global memory follows from what these warps load.
         for (int n0 = 0; a + kAuxWarps * n0 < n_items; n0 += 32) {
             int slot = -1, len = 0, flags = kMetaSkip, item = 0;
             float gs = 0.f, bt = 0.f;
@@ -383,11 +412,7 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     slot = -1;
                 }
             }
-            if (!waited) {
-                asm volatile("griddepcontrol.wait;\n" ::: "memory");
-                waited = true;
-            }
-            if (slot >= 0) {
+            if (slot >= 0) {   // (these warps have waited for the preceding kernel in the prologue)
                 if (!kVecDecay && tk.g) gs = tk.g[item];  // no gate: plain linear attention
                 if (kDelta) bt = tk.beta[item];
                 len = st.log_len[(size_t)slot * H + item % H];

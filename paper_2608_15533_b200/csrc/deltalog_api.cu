@@ -181,37 +181,43 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
     // hand-over slots: two while the base tile's arrival sets the pace; with a 16-bit base the chain
     // prep -> stream -> epilogue is the longer one and four units are kept in flight
     static const int env_slots = env_int("DELTALOG_PIPE_SLOTS", 0);
-    PipeCfg cfg{0, 0, env_slots == 4 ? 2 : env_slots == 2 ? 1 : (sizeof(BT) == 2 ? 2 : 1), -1};
+    PipeCfg cfg{0, 0, env_slots == 4 ? 2 : env_slots == 2 ? 1 : (sizeof(BT) == 2 ? 2 : 1), -1};  // depths set below
 #if DELTALOG_TEST_HOOKS
     cfg.test_drop_item = env_int_now("DELTALOG_TEST_DROP_ITEM", -1);
 #endif
     int ctas = env_ctas > 0 ? env_ctas : 1;
     if (pipelined) {
-        const int aux = AuxLayout<OP, D, IO, UL>(st.cap).bytes;
+        // Shared memory of a CTA: barriers, hand-over slots, the base ring (its place is fixed, so that its
+        // producers can start at once) and the region of the aux ring, whose stages the kernel sizes by the
+        // longest live log among the CTA's units.  The region must hold two stages in the worst case (logs one
+        // short of full); the base ring takes what is left, up to the depth that saturates HBM (fp32 base:
+        // 128 KiB in flight per SM; 16-bit base: units pass twice as fast, a somewhat shorter ring and more aux
+        // stages).  Each chunk of a tile has its own producer warp, which refills a stage as soon as THAT chunk
+        // has been consumed; a warp's successive chunks are kChunks apart in the ring, so with fewer than kChunks
+        // stages it would wait for a phase of the stage's barrier that it cannot tell from the one before
+        // (one-bit parity): the ring must hold at least one whole tile, otherwise one CTA per unit it is.
+        const int worst = 2 * AuxLayout<OP, D, IO, UL>(st.cap).bytes;
         const int fixed = kPipeBarrierBytes + pipe_scratch_bytes<D>(cfg.slot_shift);
-        // fp32 base: 128 KiB of base tiles in flight per SM saturate HBM, four aux stages (two are held by
-        // the scalar groups, the rest is prefetch).  16-bit base: units pass twice as fast and up to four sit
-        // between the prep and the epilogue group, so more aux stages and a somewhat shorter base ring.
         const bool b16 = sizeof(BT) == 2;
-        const int want_base = env_base > 0 ? env_base : (b16 ? 5 : 8) * (kChunkBytes / kStage);
-        const int want_aux = env_aux > 0 ? env_aux : (b16 ? 6 : 4);
+        int want_base = env_base > 0 ? env_base : (b16 ? 5 : 8) * (kChunkBytes / kStage);
+        if (want_base < kChunks) want_base = kChunks;
+        if (want_base > kPipeMaxBase) want_base = kPipeMaxBase;
+        const int min_aux = env_aux > 0 ? env_aux : (b16 ? 6 : 4);   // aux stages wanted at the full capacity ...
         for (; ctas >= 1; --ctas) {
             int budget = dev.smem_per_sm / ctas - 1024;
             if (budget > dev.smem_optin) budget = dev.smem_optin;
-            // aux stages: two are held by the scalar group (unit i and i+1), the rest is prefetch
-            for (cfg.n_aux = want_aux; cfg.n_aux >= 2; --cfg.n_aux) {
-                cfg.n_base = (budget - fixed - cfg.n_aux * aux) / kStage;
-                if (cfg.n_base >= want_base || cfg.n_aux == 2) break;
+            // ... as long as the base ring keeps its depth; at least the two stages of the worst case
+            int aux_want = min_aux * (worst / 2);
+            if (aux_want > budget - fixed - want_base * kStage) aux_want = budget - fixed - want_base * kStage;
+            if (aux_want < worst) aux_want = worst;
+            cfg.n_base = (budget - fixed - aux_want) / kStage;
+            if (cfg.n_base > want_base) cfg.n_base = want_base;
+            if (cfg.n_base >= kChunks) {
+                cfg.aux_bytes = (budget - fixed - cfg.n_base * kStage) / 128 * 128;
+                break;
             }
-            // Each chunk of a tile has its own producer warp, which refills a stage as soon as THAT chunk has
-            // been consumed; a warp's successive chunks are kChunks apart in the ring, so with fewer than
-            // kChunks stages it would wait for a phase of the stage's barrier that it cannot tell from the
-            // one before (one-bit parity).  The ring must hold at least one whole tile.
-            if (cfg.n_base >= kChunks) break;
         }
-        if (ctas < 1) pipelined = false;  // the aux stages leave no room for a tile: one CTA per unit instead
-        if (cfg.n_base > 8 * (kChunkBytes / kStage)) cfg.n_base = 8 * (kChunkBytes / kStage);
-        if (env_base > 0 && cfg.n_base > env_base) cfg.n_base = env_base > kChunks ? env_base : kChunks;
+        if (ctas < 1) pipelined = false;
     }
     if (pipelined) {
         // What L2 holds on to across steps is about half its size on this part (measured: a re-read set is
@@ -224,7 +230,7 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
         const float full_log = (float)total * (float)st.cap * entry;
         st.l2_pin_bytes = pin_mb >= 0 ? pin_mb * kMiB : fminf(24.f * kMiB, fmaxf(0.f, 64.f * kMiB - 0.75f * full_log));
         auto kernel = decode_pipelined_kernel<OP, D, IO, UL, BT>;
-        const int smem = pipe_smem_bytes<OP, D, IO, UL, BT>(st.cap, cfg);
+        const int smem = pipe_smem_bytes<D, BT>(cfg);
         if (int rc = ensure_smem(kernel, smem)) return rc;
         const int grid = total < dev.sms * ctas ? total : dev.sms * ctas;
         if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, grid, kPipeThreads, smem, stream, st, tk, cfg);
