@@ -37,7 +37,9 @@
  *     range) make the kernel skip that row, OR a bit into *state->status (if non-NULL) and carry
  *     on; kernels never trap.  Rows with slot index < 0 are padding and are skipped silently.
  *   - The same slot must not appear twice in one call.
- *   - Supported shapes: d_k == d_v in {64, 128}; 1 <= cap <= 64; klog_dtype == io_dtype;
+ *   - Supported shapes: d_k and d_v each 64 or 128 (they may differ: the tile is d_k rows x d_v columns;
+ *     q, k, the gate of the per-key operators and K_log are d_k wide, v, out and U_log d_v wide);
+ *     1 <= cap <= 64; klog_dtype == io_dtype;
  *     ulog_dtype == io_dtype for the operators with b_t = v_t; F32 for GDN / KDA (the paper keeps b_t in
  *     fp32 against cancellation in the correction path), or, as a reduced-precision variant that does
  *     NOT meet the 1e-4 state tolerance, == io_dtype == BF16.

@@ -16,9 +16,9 @@ constexpr int kWarps = kThreads / 32;
 #ifndef DELTALOG_MAT_THREADS
 #define DELTALOG_MAT_THREADS 256
 #endif
-template <int D>
+template <int DK, int DV>
 __host__ __device__ constexpr int mat_threads() {
-    return D >= 128 ? DELTALOG_MAT_THREADS : 256;
+    return (DK >= 128 && DV >= 128) ? DELTALOG_MAT_THREADS : 256;
 }
 constexpr int kMaxCap = 64;
 

@@ -17,25 +17,27 @@
 
 namespace deltalog {
 
-// Threads per CTA: 256 at head size 128; 128 at head size 64, where the tile is only 16 KiB and the
-// run time of a CTA is one long latency chain (length -> snapshot and log -> coefficients): smaller
-// CTAs let eight of them overlap their chains on an SM instead of four.
-template <int D>
+// Threads per CTA: 256 when a head dimension is 128; 128 at head size 64 x 64, where the tile is only
+// 16 KiB and the run time of a CTA is one long latency chain (length -> snapshot and log -> coefficients):
+// smaller CTAs let eight of them overlap their chains on an SM instead of four.  (The key dimension DK
+// indexes the tile's rows, the value dimension DV its columns; they may differ.)
+template <int DK, int DV>
 __host__ __device__ constexpr int decode_threads() {
-    return D >= 128 ? 256 : 128;
+    return (DK >= 128 || DV >= 128) ? 256 : 128;
 }
 
-template <int D, typename IO, typename UL>
+template <int DK, int DV, typename IO, typename UL>
 __host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
-    const size_t dl = (op == DELTALOG_GDN || op == DELTALOG_RETNET || op == DELTALOG_LINATTN) ? 1 : D;
+    const size_t dl = (op == DELTALOG_GDN || op == DELTALOG_RETNET || op == DELTALOG_LINATTN) ? 1 : DK;
     size_t bytes = 0;
-    bytes += sizeof(float) * D * 5;                 // q, k (raw), mul_k, mul_q, lbar'/u scratch
-    bytes += sizeof(float) * D;                     // lbar_old (vector ops)
+    bytes += sizeof(float) * DK * 4;                // q, k (raw), mul_k, mul_q
+    bytes += sizeof(float) * DV;                    // b
+    bytes += sizeof(float) * DK;                    // lbar_old (vector ops)
     bytes += sizeof(float) * 2 * kMaxCap;           // replay coefficients
-    bytes += sizeof(float) * 2 * D * (decode_threads<D>() / (D / 4));  // cross-row-lane partial sums
+    bytes += sizeof(float) * 2 * DV * (decode_threads<DK, DV>() / (DV / 4));  // cross-row-lane partial sums
     bytes += 16;                                    // scalars
-    bytes += sizeof(UL) * (size_t)cap * D;          // U log
-    bytes += sizeof(IO) * (size_t)cap * D;          // K log
+    bytes += sizeof(UL) * (size_t)cap * DV;         // U log
+    bytes += sizeof(IO) * (size_t)cap * DK;         // K log
     bytes += sizeof(float) * (((size_t)cap * dl + 3) / 4 * 4);  // Lambda log
     return bytes;
 }
@@ -43,18 +45,20 @@ __host__ __device__ constexpr size_t decode_smem_bytes(int op, int cap) {
 #ifndef DELTALOG_SIMPLE_CTAS
 #define DELTALOG_SIMPLE_CTAS 2
 #endif
-template <int OP, int D, typename IO, typename UL, typename BT = float>
-__global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPLE_CTAS : 8) decode_append_kernel(StateArgs st, TokenArgs tk) {
-    constexpr int NT = decode_threads<D>();
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT = float>
+__global__ void __launch_bounds__(decode_threads<DK, DV>(), decode_threads<DK, DV>() >= 256 ? DELTALOG_SIMPLE_CTAS : 8)
+decode_append_kernel(StateArgs st, TokenArgs tk) {
+    constexpr int NT = decode_threads<DK, DV>();
     constexpr int NW = NT / 32;
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
-    constexpr int DL = kVecDecay ? D : 1;
-    constexpr int C4 = D / 4;          // float4 columns per state row
+    constexpr int DL = kVecDecay ? DK : 1;
+    constexpr int C4 = DV / 4;         // float4 columns per state row
     constexpr int RL = NT / C4;        // rows covered by one pass of the CTA
-    constexpr int NP = D / RL;         // passes over the tile
-    constexpr int EPL = D / 32;        // key elements per lane in a warp-wide dot product
+    constexpr int NP = DK / RL;        // passes over the tile
+    constexpr int EPL = DK / 32;       // key elements per lane in a warp-wide dot product
+    static_assert(NT >= DK && NT >= (kDelta ? 2 : 1) * DV, "one thread per key channel and per output column");
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
@@ -68,7 +72,7 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     const int cap = st.cap;
 
     // ---- 1. request the whole base tile (independent of every other load) -------------------
-    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * D * D;
+    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * DK * DV;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
@@ -88,39 +92,39 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *q_s = reinterpret_cast<float *>(smem_raw);
-    float *k_s = q_s + D;
-    float *mk_s = k_s + D;      // e^{lbar'} . k
-    float *mq_s = mk_s + D;     // e^{lbar'} . q   (RWKV6: e^{lbar} . r)
-    float *b_s = mq_s + D;      // value-side factor, shared between the two output halves
-    float *lold_s = b_s + D;    // lbar (vector-decay ops)
-    float *ck_s = lold_s + D;   // [kMaxCap]
+    float *k_s = q_s + DK;
+    float *mk_s = k_s + DK;     // e^{lbar'} . k
+    float *mq_s = mk_s + DK;    // e^{lbar'} . q   (RWKV6: e^{lbar} . r)
+    float *b_s = mq_s + DK;     // [DV] value-side factor, shared between the two output halves
+    float *lold_s = b_s + DV;   // lbar (vector-decay ops)
+    float *ck_s = lold_s + DK;  // [kMaxCap]
     float *cq_s = ck_s + kMaxCap;
-    float *red_s = cq_s + kMaxCap;           // [RL][2][D]
-    float *scal_s = red_s + 2 * D * RL;      // [0] = q.k  (or r.(bonus.k))
+    float *red_s = cq_s + kMaxCap;           // [RL][2][DV]
+    float *scal_s = red_s + 2 * DV * RL;     // [0] = q.k  (or r.(bonus.k))
     UL *U_s = reinterpret_cast<UL *>(scal_s + 4);
-    IO *K_s = reinterpret_cast<IO *>(U_s + (size_t)cap * D);
-    float *Lam_s = reinterpret_cast<float *>(K_s + (size_t)cap * D);
+    IO *K_s = reinterpret_cast<IO *>(U_s + (size_t)cap * DV);
+    float *Lam_s = reinterpret_cast<float *>(K_s + (size_t)cap * DK);
 
     // ---- 2. stage the live log entries (asynchronously) and the token vectors ---------------
-    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
-    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * DK;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * DV;
     const float *Lg = st.decay_log + unit * cap * DL;
-    constexpr int kEntryBytes = D * (int)(sizeof(IO) + sizeof(UL)) + DL * 4;
+    constexpr int kEntryBytes = DK * (int)sizeof(IO) + DV * (int)sizeof(UL) + DL * 4;
     const int total_units = tk.B * st.H;
     const uint64_t keep_rd = l2_policy_keep(st.keep_fraction(len, total_units, kEntryBytes));
-    cta_cp_async_hint(K_s, Kg, len * D * (int)sizeof(IO), tid, NT, keep_rd);
-    cta_cp_async_hint(U_s, Ug, len * D * (int)sizeof(UL), tid, NT, keep_rd);
-    if (kVecDecay) cta_cp_async_hint(Lam_s, Lg, len * D * (int)sizeof(float), tid, NT, keep_rd);
+    cta_cp_async_hint(K_s, Kg, len * DK * (int)sizeof(IO), tid, NT, keep_rd);
+    cta_cp_async_hint(U_s, Ug, len * DV * (int)sizeof(UL), tid, NT, keep_rd);
+    if (kVecDecay) cta_cp_async_hint(Lam_s, Lg, len * DK * (int)sizeof(float), tid, NT, keep_rd);
     cp_async_commit();
     if (!kVecDecay && tid < len) Lam_s[tid] = Lg[tid];
 
-    const IO *qg = static_cast<const IO *>(tk.q) + tk.qk_row(b, h) * D;
-    const IO *kg = static_cast<const IO *>(tk.k) + tk.qk_row(b, h) * D;
-    const IO *vg = static_cast<const IO *>(tk.v) + row * D;
+    const IO *qg = static_cast<const IO *>(tk.q) + tk.qk_row(b, h) * DK;
+    const IO *kg = static_cast<const IO *>(tk.k) + tk.qk_row(b, h) * DK;
+    const IO *vg = static_cast<const IO *>(tk.v) + row * DV;
     const float *gg = tk.g + row * DL;
     IO k_raw = from_f32<IO>(0.f);
     float lnew = 0.f;
-    if (tid < D) {
+    if (tid < DK) {
         const float qv = to_f32(qg[tid]);
         k_raw = kg[tid];
         const float kv = to_f32(k_raw);
@@ -142,8 +146,8 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            float kij = to_f32(K_s[i * D + j]);
-            if (kVecDecay) kij *= expf(lold_s[j] - Lam_s[i * D + j]);
+            float kij = to_f32(K_s[i * DK + j]);
+            if (kVecDecay) kij *= expf(lold_s[j] - Lam_s[i * DK + j]);
             dq = fmaf(q_s[j], kij, dq);
             if (kDelta) dk = fmaf(k_s[j], kij, dk);
         }
@@ -160,7 +164,7 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * DK + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -181,22 +185,22 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
     __syncthreads();
 
     // ---- 5. reduce, replay the value-side log, form b and the output, append ----------------
-    const int which = tid / D, c = tid % D;  // which: 0 -> y_k half, 1 -> y_q half
+    const int which = tid / DV, c = tid % DV;  // which: 0 -> y_k half, 1 -> y_q half
     float y = 0.f;
-    const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+    const bool active = kDelta ? (tid < 2 * DV) : (tid < DV);
     const int sel = kDelta ? which : 1;
     if (active) {
 #pragma unroll
-        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * DV + c];
         const float *coef = sel ? cq_s : ck_s;
-        for (int i = 0; i < len; ++i) y = fmaf(coef[i], to_f32(U_s[i * D + c]), y);
+        for (int i = 0; i < len; ++i) y = fmaf(coef[i], to_f32(U_s[i * DV + c]), y);
     }
-    UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * D;
-    IO *og = static_cast<IO *>(tk.out) + row * D;
+    UL *Uout = static_cast<UL *>(st.U_log) + (unit * cap + len) * DV;
+    IO *og = static_cast<IO *>(tk.out) + row * DV;
     // the new entry is read again by the following steps: same L2 policy as the log's reads
     const uint64_t keep_wr = l2_policy_keep(st.keep_fraction(len + 1, total_units, kEntryBytes));
     if (kDelta) {
-        if (tid < D) {
+        if (tid < DV) {
             const float bval = tk.beta[row] * (to_f32(vg[c]) - y);
             b_s[c] = bval;
             st_hint(Uout + c, from_f32<UL>(bval), keep_wr);
@@ -208,8 +212,8 @@ __global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? DELTALOG_SIMPL
         og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], to_f32(v_raw), y));
         st_hint(Uout + c, from_f32<UL>(to_f32(v_raw)), keep_wr);  // lossless: U log dtype equals the I/O dtype
     }
-    if (tid < D) {
-        st_hint(static_cast<IO *>(st.K_log) + (unit * cap + len) * D + tid, k_raw, keep_wr);
+    if (tid < DK) {
+        st_hint(static_cast<IO *>(st.K_log) + (unit * cap + len) * DK + tid, k_raw, keep_wr);
         if (kVecDecay) st_hint(st.decay_log + (unit * cap + len) * DL + tid, lnew, keep_wr);
     }
     if (tid == 0) {

@@ -19,16 +19,16 @@
 
 namespace deltalog {
 
-template <int OP, int D, typename IO, typename UL, typename BT = float>
-__global__ void __launch_bounds__(decode_threads<D>(), D >= 128 ? 2 : 8)
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT = float>
+__global__ void __launch_bounds__(decode_threads<DK, DV>(), decode_threads<DK, DV>() >= 256 ? 2 : 8)
 decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
-    constexpr int NT = decode_threads<D>();
+    constexpr int NT = decode_threads<DK, DV>();
     constexpr int NW = NT / 32;
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
-    constexpr int DL = kVecDecay ? D : 1;
-    constexpr int C4 = D / 4, RL = NT / C4, NP = D / RL, EPL = D / 32;
+    constexpr int DL = kVecDecay ? DK : 1;
+    constexpr int C4 = DV / 4, RL = NT / C4, NP = DK / RL, EPL = DK / 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
@@ -38,7 +38,7 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
     const int cap = st.cap;
 
     // ---- the base tile: one read for all T tokens ------------------------------------------------
-    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * D * D;
+    const BT *Sg = static_cast<const BT *>(st.S_base) + unit * DK * DV;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
@@ -52,26 +52,26 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *q_s = reinterpret_cast<float *>(smem_raw);
-    float *k_s = q_s + D;
-    float *mk_s = k_s + D;      // e^{lbar'} . k
-    float *mq_s = mk_s + D;     // e^{lbar'} . q   (RWKV6: e^{lbar} . r)
-    float *b_s = mq_s + D;
-    float *lold_s = b_s + D;    // the decay level the readouts refer to
-    float *ck_s = lold_s + D;   // [kMaxCap]
+    float *k_s = q_s + DK;
+    float *mk_s = k_s + DK;     // e^{lbar'} . k
+    float *mq_s = mk_s + DK;    // e^{lbar'} . q   (RWKV6: e^{lbar} . r)
+    float *b_s = mq_s + DK;     // [DV]
+    float *lold_s = b_s + DV;   // the decay level the readouts refer to
+    float *ck_s = lold_s + DK;  // [kMaxCap]
     float *cq_s = ck_s + kMaxCap;
-    float *red_s = cq_s + kMaxCap;           // [RL][2][D]
-    float *scal_s = red_s + 2 * D * RL;      // [0] = q.k  (or r.(bonus.k))
+    float *red_s = cq_s + kMaxCap;           // [RL][2][DV]
+    float *scal_s = red_s + 2 * DV * RL;     // [0] = q.k  (or r.(bonus.k))
     UL *U_s = reinterpret_cast<UL *>(scal_s + 4);
-    IO *K_s = reinterpret_cast<IO *>(U_s + (size_t)cap * D);
-    float *Lam_s = reinterpret_cast<float *>(K_s + (size_t)cap * D);
+    IO *K_s = reinterpret_cast<IO *>(U_s + (size_t)cap * DV);
+    float *Lam_s = reinterpret_cast<float *>(K_s + (size_t)cap * DK);
 
     // ---- the live log, staged once; it grows in shared memory below ------------------------------
-    IO *Kg = static_cast<IO *>(st.K_log) + unit * cap * D;
-    UL *Ug = static_cast<UL *>(st.U_log) + unit * cap * D;
+    IO *Kg = static_cast<IO *>(st.K_log) + unit * cap * DK;
+    UL *Ug = static_cast<UL *>(st.U_log) + unit * cap * DV;
     float *Lg = st.decay_log + unit * cap * DL;
-    cta_cp_async(K_s, Kg, len0 * D * (int)sizeof(IO), tid, NT);
-    cta_cp_async(U_s, Ug, len0 * D * (int)sizeof(UL), tid, NT);
-    if (kVecDecay) cta_cp_async(Lam_s, Lg, len0 * D * (int)sizeof(float), tid, NT);
+    cta_cp_async(K_s, Kg, len0 * DK * (int)sizeof(IO), tid, NT);
+    cta_cp_async(U_s, Ug, len0 * DV * (int)sizeof(UL), tid, NT);
+    if (kVecDecay) cta_cp_async(Lam_s, Lg, len0 * DK * (int)sizeof(float), tid, NT);
     cp_async_commit();
     if (!kVecDecay && tid < len0) Lam_s[tid] = Lg[tid];
     cp_async_wait_all();
@@ -87,16 +87,16 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
         Tok x;
         const size_t row = ((size_t)b * T + t) * st.H + h;                       // (batch row, token, head)
         const size_t row_qk = ((size_t)b * T + t) * tk.H_qk + h / tk.qk_group;
-        const int c = tid % D;
+        const int c = tid % DV;
         x.q = x.k = from_f32<IO>(0.f);
-        x.g = x.beta = 0.f;
-        if (tid < D) {
-            x.q = static_cast<const IO *>(tk.q)[row_qk * D + tid];
-            x.k = static_cast<const IO *>(tk.k)[row_qk * D + tid];
+        x.g = 0.f;
+        x.beta = kDelta ? tk.beta[row] : 0.f;
+        if (tid < DK) {
+            x.q = static_cast<const IO *>(tk.q)[row_qk * DK + tid];
+            x.k = static_cast<const IO *>(tk.k)[row_qk * DK + tid];
             x.g = tk.g ? tk.g[row * DL + (kVecDecay ? tid : 0)] : 0.f;
-            if (kDelta) x.beta = tk.beta[row];
         }
-        x.v = static_cast<const IO *>(tk.v)[row * D + c];
+        x.v = static_cast<const IO *>(tk.v)[row * DV + c];
         return x;
     };
     Tok nxt = load_token(0);
@@ -107,7 +107,7 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
         if (t + 1 < T) nxt = load_token(t + 1);
         IO k_raw = cur.k;
         float lnew = 0.f;
-        if (tid < D) {
+        if (tid < DK) {
             const float qv = to_f32(cur.q);
             const float kv = to_f32(k_raw);
             const float lold = (len > 0) ? Lam_s[(size_t)(len - 1) * DL + (kVecDecay ? tid : 0)] : 0.f;
@@ -127,8 +127,8 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
 #pragma unroll
             for (int e = 0; e < EPL; ++e) {
                 const int j = lane + 32 * e;
-                float kij = to_f32(K_s[i * D + j]);
-                if (kVecDecay) kij *= expf(lold_s[j] - Lam_s[i * D + j]);
+                float kij = to_f32(K_s[i * DK + j]);
+                if (kVecDecay) kij *= expf(lold_s[j] - Lam_s[i * DK + j]);
                 dq = fmaf(q_s[j], kij, dq);
                 if (kDelta) dk = fmaf(k_s[j], kij, dk);
             }
@@ -145,7 +145,7 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
 #pragma unroll
             for (int e = 0; e < EPL; ++e) {
                 const int j = lane + 32 * e;
-                const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
+                const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * DK + j];
                 d = fmaf(q_s[j] * w, k_s[j], d);
             }
             d = warp_sum(d);
@@ -166,24 +166,24 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
         __syncthreads();
 
         // reduce, value-side replay, b, output, append (shared memory and global)
-        const int which = tid / D, c = tid % D;
-        const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+        const int which = tid / DV, c = tid % DV;
+        const bool active = kDelta ? (tid < 2 * DV) : (tid < DV);
         const int sel = kDelta ? which : 1;
         float y = 0.f;
         if (active) {
 #pragma unroll
-            for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+            for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * DV + c];
             const float *coef = sel ? cq_s : ck_s;
-            for (int i = 0; i < len; ++i) y = fmaf(coef[i], to_f32(U_s[i * D + c]), y);
+            for (int i = 0; i < len; ++i) y = fmaf(coef[i], to_f32(U_s[i * DV + c]), y);
         }
-        IO *og = static_cast<IO *>(tk.out) + row * D;
+        IO *og = static_cast<IO *>(tk.out) + row * DV;
         if (kDelta) {
-            if (tid < D) {
+            if (tid < DV) {
                 const float bval = cur.beta * (to_f32(cur.v) - y);
                 b_s[c] = bval;
                 const UL bu = from_f32<UL>(bval);
-                U_s[(size_t)len * D + c] = bu;
-                Ug[(size_t)len * D + c] = bu;
+                U_s[(size_t)len * DV + c] = bu;
+                Ug[(size_t)len * DV + c] = bu;
             }
             __syncthreads();
             if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
@@ -191,15 +191,15 @@ decode_multi_kernel(StateArgs st, TokenArgs tk, int32_t T) {
             const IO v_raw = cur.v;
             og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], to_f32(v_raw), y));
             const UL bu = from_f32<UL>(to_f32(v_raw));
-            U_s[(size_t)len * D + c] = bu;
-            Ug[(size_t)len * D + c] = bu;
+            U_s[(size_t)len * DV + c] = bu;
+            Ug[(size_t)len * DV + c] = bu;
         }
-        if (tid < D) {
-            K_s[(size_t)len * D + tid] = k_raw;
-            Kg[(size_t)len * D + tid] = k_raw;
+        if (tid < DK) {
+            K_s[(size_t)len * DK + tid] = k_raw;
+            Kg[(size_t)len * DK + tid] = k_raw;
             if (kVecDecay) {
-                Lam_s[(size_t)len * D + tid] = lnew;
-                Lg[(size_t)len * D + tid] = lnew;
+                Lam_s[(size_t)len * DK + tid] = lnew;
+                Lg[(size_t)len * DK + tid] = lnew;
             }
         }
         if (tid == 0 && !kVecDecay) {

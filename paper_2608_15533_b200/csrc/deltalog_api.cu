@@ -161,9 +161,14 @@ const DeviceInfo &device_info() {
 // Tuning knobs (environment, read once): DELTALOG_DECODE_IMPL = 0 auto | 1 one-CTA-per-unit | 2 pipelined;
 // DELTALOG_CTAS_PER_SM, DELTALOG_BASE_STAGES, DELTALOG_AUX_STAGES override the pipelined kernel's shape.
 
-template <int OP, int D, typename IO, typename UL, typename BT>
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stream) {
     StateArgs st = st_in;
+    const int total_units = tk.B * st.H;
+    // The persistent kernels are built for square tiles (head size 128, and 64 with an fp32 base); other
+    // shapes (d_k != d_v) run one CTA per unit.
+    if constexpr (DK == DV) {
+    constexpr int D = DK;
     static const int impl = env_int("DELTALOG_DECODE_IMPL", 0);
     static const int env_ctas = env_int("DELTALOG_CTAS_PER_SM", 0);
     static const int env_base = env_int("DELTALOG_BASE_STAGES", 0);
@@ -261,24 +266,26 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
             return finish_launch();
         }
     }
-    auto kernel = decode_append_kernel<OP, D, IO, UL, BT>;
-    const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
+    }
+    auto kernel = decode_append_kernel<OP, DK, DV, IO, UL, BT>;
+    const size_t smem = decode_smem_bytes<DK, DV, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED) return launch_chained(kernel, total, decode_threads<D>(), smem, stream, st, tk);
-    kernel<<<total, decode_threads<D>(), smem, stream>>>(st, tk);
+    if (tk.hints & DELTALOG_HINT_BASE_UNTOUCHED)
+        return launch_chained(kernel, total_units, decode_threads<DK, DV>(), smem, stream, st, tk);
+    kernel<<<total_units, decode_threads<DK, DV>(), smem, stream>>>(st, tk);
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL, typename BT>
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_decode_multi(const StateArgs &st, const TokenArgs &tk, int32_t T, cudaStream_t stream) {
-    auto kernel = decode_multi_kernel<OP, D, IO, UL, BT>;
-    const size_t smem = decode_smem_bytes<D, IO, UL>(OP, st.cap);
+    auto kernel = decode_multi_kernel<OP, DK, DV, IO, UL, BT>;
+    const size_t smem = decode_smem_bytes<DK, DV, IO, UL>(OP, st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<tk.B * st.H, decode_threads<D>(), smem, stream>>>(st, tk, T);
+    kernel<<<tk.B * st.H, decode_threads<DK, DV>(), smem, stream>>>(st, tk, T);
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL, typename BT>
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_t only_if_full,
                  cudaStream_t stream) {
     // DELTALOG_MERGE_TC = 1 (head size 128, no predicate): the contraction over the log entries runs
@@ -288,7 +295,7 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
     // (measured on configuration 1: 110 / 119 / 142 / 215 us at capacity 4 / 16 / 32 / 64 against
     // 85 / 99 / 130 / 195 us for the packed-FMA kernel).
     static const int use_tc = env_int("DELTALOG_MERGE_TC", 0);
-    if constexpr (D == kTcD && std::is_same<BT, float>::value) {
+    if constexpr (DK == kTcD && DV == kTcD && std::is_same<BT, float>::value) {
         if (use_tc && !only_if_full) {
             auto kernel = merge_tc_kernel<OP, IO, UL>;
             const size_t bytes = merge_tc_smem_bytes<OP, IO, UL>(st.cap);
@@ -297,88 +304,94 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
             return finish_launch();
         }
     }
-    const size_t smem = merge_smem_bytes<D>(st.cap);
+    const size_t smem = merge_smem_bytes<DK, DV>(st.cap);
     // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
     // call over a whole batch whose fills are staggered) most units are skipped: kMergePack candidates per CTA.
     const int pairs = n * st.H;
     if (only_if_full) {
-        auto kernel = merge_kernel<OP, D, IO, UL, kMergePack, BT>;
+        auto kernel = merge_kernel<OP, DK, DV, IO, UL, kMergePack, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
-        kernel<<<(pairs + kMergePack - 1) / kMergePack, mat_threads<D>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
+        kernel<<<(pairs + kMergePack - 1) / kMergePack, mat_threads<DK, DV>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
     } else {
-        auto kernel = merge_kernel<OP, D, IO, UL, 1, BT>;
+        auto kernel = merge_kernel<OP, DK, DV, IO, UL, 1, BT>;
         if (int rc = ensure_smem(kernel, smem)) return rc;
-        kernel<<<pairs, mat_threads<D>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
+        kernel<<<pairs, mat_threads<DK, DV>(), smem, stream>>>(st, slot_idx, only_if_full, pairs);
     }
     return finish_launch();
 }
 
-template <int OP, int D, typename IO, typename UL, typename BT>
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    auto kernel = decode_merge_step_kernel<OP, D, IO, UL, BT>;
-    const size_t smem = fused_step_smem_bytes<D>(st.cap);
+    auto kernel = decode_merge_step_kernel<OP, DK, DV, IO, UL, BT>;
+    const size_t smem = fused_step_smem_bytes<DK, DV>(st.cap);
     if (int rc = ensure_smem(kernel, smem)) return rc;
-    kernel<<<tk.B * st.H, mat_threads<D>(), smem, stream>>>(st, tk);
+    kernel<<<tk.B * st.H, mat_threads<DK, DV>(), smem, stream>>>(st, tk);
     return finish_launch();
 }
 
-template <int OP, int D, typename IO>
+template <int OP, int DK, int DV, typename IO>
 int launch_eager(void *S, const deltalog_desc *d, int32_t *status, const TokenArgs &tk, cudaStream_t stream) {
     if constexpr (!std::is_same<IO, float>::value) {
         if (d->base_dtype == DELTALOG_BF16) {
-            eager_step_kernel<OP, D, IO, __nv_bfloat16>
+            eager_step_kernel<OP, DK, DV, IO, __nv_bfloat16>
                 <<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
             return finish_launch();
         }
     }
-    eager_step_kernel<OP, D, IO, float><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
+    eager_step_kernel<OP, DK, DV, IO, float><<<tk.B * d->H, kThreads, 0, stream>>>(S, d->num_slots, d->H, d->scale, status, tk);
     return finish_launch();
 }
 
-// Expand (op, d, io dtype) into the template instantiation and call F<OP, D, IO>::run(args...).
+// Expand (op, d_k, d_v, io dtype) into the template instantiation: CALL(OP, DK, DV, IO).
 #define DELTALOG_DISPATCH(desc, CALL)                                                        \
     do {                                                                                     \
-        const int op_ = (desc)->op, d_ = (desc)->d_k, io_ = (desc)->io_dtype;                \
+        const int op_ = (desc)->op, dk_ = (desc)->d_k, dv_ = (desc)->d_v, io_ = (desc)->io_dtype; \
         if (op_ == DELTALOG_GDN) {                                                           \
-            DELTALOG_DISPATCH_D(DELTALOG_GDN, d_, io_, CALL);                                \
+            DELTALOG_DISPATCH_D(DELTALOG_GDN, dk_, dv_, io_, CALL);                          \
         } else if (op_ == DELTALOG_KDA) {                                                    \
-            DELTALOG_DISPATCH_D(DELTALOG_KDA, d_, io_, CALL);                                \
+            DELTALOG_DISPATCH_D(DELTALOG_KDA, dk_, dv_, io_, CALL);                          \
         } else if (op_ == DELTALOG_RETNET || op_ == DELTALOG_LINATTN) {                      \
-            DELTALOG_DISPATCH_D(DELTALOG_RETNET, d_, io_, CALL); /* linear attention: null gate */ \
+            DELTALOG_DISPATCH_D(DELTALOG_RETNET, dk_, dv_, io_, CALL); /* linear attention: null gate */ \
         } else if (op_ == DELTALOG_GLA) {                                                    \
-            DELTALOG_DISPATCH_D(DELTALOG_GLA, d_, io_, CALL);                                \
+            DELTALOG_DISPATCH_D(DELTALOG_GLA, dk_, dv_, io_, CALL);                          \
         } else {                                                                             \
-            DELTALOG_DISPATCH_D(DELTALOG_RWKV6, d_, io_, CALL);                              \
+            DELTALOG_DISPATCH_D(DELTALOG_RWKV6, dk_, dv_, io_, CALL);                        \
         }                                                                                    \
     } while (0)
-#define DELTALOG_DISPATCH_D(OP, d_, io_, CALL)                                               \
-    if (d_ == 64) {                                                                          \
-        if (io_ == DELTALOG_F32) { CALL(OP, 64, float); } else { CALL(OP, 64, __nv_bfloat16); } \
+#define DELTALOG_DISPATCH_D(OP, dk_, dv_, io_, CALL)                                         \
+    if (dk_ == 64 && dv_ == 64) {                                                            \
+        DELTALOG_DISPATCH_IO(OP, 64, 64, io_, CALL);                                         \
+    } else if (dk_ == 128 && dv_ == 128) {                                                   \
+        DELTALOG_DISPATCH_IO(OP, 128, 128, io_, CALL);                                       \
+    } else if (dk_ == 128) {                                                                 \
+        DELTALOG_DISPATCH_IO(OP, 128, 64, io_, CALL);                                        \
     } else {                                                                                 \
-        if (io_ == DELTALOG_F32) { CALL(OP, 128, float); } else { CALL(OP, 128, __nv_bfloat16); } \
+        DELTALOG_DISPATCH_IO(OP, 64, 128, io_, CALL);                                        \
     }
+#define DELTALOG_DISPATCH_IO(OP, DK, DV, io_, CALL)                                          \
+    if (io_ == DELTALOG_F32) { CALL(OP, DK, DV, float); } else { CALL(OP, DK, DV, __nv_bfloat16); }
 
 // The value-side log keeps the I/O dtype where b = v (lossless).  For the delta rule it is fp32 by
 // default; a 16-bit U log (descriptor ulog_dtype == io_dtype == BF16) is the reduced-precision variant.
 // The dense base is fp32 unless the descriptor asks for the 16-bit state (16-bit I/O only).
-#define DELTALOG_WITH_UL(OP, IO, desc, FN, D, ...)                                                         \
+#define DELTALOG_WITH_UL(OP, IO, desc, FN, DK, DV, ...)                                                    \
     do {                                                                                                  \
         if constexpr (!std::is_same<IO, float>::value) {                                                  \
             if ((desc)->base_dtype == DELTALOG_BF16) {                                                    \
-                DELTALOG_WITH_UL_BT(OP, IO, __nv_bfloat16, desc, FN, D, __VA_ARGS__);                     \
+                DELTALOG_WITH_UL_BT(OP, IO, __nv_bfloat16, desc, FN, DK, DV, __VA_ARGS__);                \
             }                                                                                             \
         }                                                                                                 \
-        DELTALOG_WITH_UL_BT(OP, IO, float, desc, FN, D, __VA_ARGS__);                                      \
+        DELTALOG_WITH_UL_BT(OP, IO, float, desc, FN, DK, DV, __VA_ARGS__);                                 \
     } while (0)
-#define DELTALOG_WITH_UL_BT(OP, IO, BT, desc, FN, D, ...)                                                  \
+#define DELTALOG_WITH_UL_BT(OP, IO, BT, desc, FN, DK, DV, ...)                                             \
     do {                                                                                                  \
         if constexpr (OpTraits<OP>::kDeltaRule) {                                                         \
             if constexpr (!std::is_same<IO, float>::value) {                                              \
-                if ((desc)->ulog_dtype != DELTALOG_F32) return FN<OP, D, IO, IO, BT>(__VA_ARGS__);         \
+                if ((desc)->ulog_dtype != DELTALOG_F32) return FN<OP, DK, DV, IO, IO, BT>(__VA_ARGS__);    \
             }                                                                                             \
-            return FN<OP, D, IO, float, BT>(__VA_ARGS__);                                                 \
+            return FN<OP, DK, DV, IO, float, BT>(__VA_ARGS__);                                            \
         } else {                                                                                          \
-            return FN<OP, D, IO, IO, BT>(__VA_ARGS__);                                                    \
+            return FN<OP, DK, DV, IO, IO, BT>(__VA_ARGS__);                                               \
         }                                                                                                 \
     } while (0)
 
@@ -400,7 +413,7 @@ int deltalog_decode_step(const deltalog_desc *desc, const deltalog_state *state,
     const StateArgs st = make_state_args(desc, state);
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_DECODE(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode, D, st, tk, s)
+#define CALL_DECODE(OP, DK, DV, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode, DK, DV, st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_DECODE);
 #undef CALL_DECODE
     return DELTALOG_ERR_INVALID_ARG;
@@ -417,7 +430,7 @@ int deltalog_decode_steps(const deltalog_desc *desc, const deltalog_state *state
     const StateArgs st = make_state_args(desc, state);
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_MULTI(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode_multi, D, st, tk, T, s)
+#define CALL_MULTI(OP, DK, DV, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_decode_multi, DK, DV, st, tk, T, s)
     DELTALOG_DISPATCH(desc, CALL_MULTI);
 #undef CALL_MULTI
     return DELTALOG_ERR_INVALID_ARG;
@@ -434,7 +447,7 @@ int deltalog_decode_merge_step(const deltalog_desc *desc, const deltalog_state *
     const StateArgs st = make_state_args(desc, state);
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_FUSED(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_fused_step, D, st, tk, s)
+#define CALL_FUSED(OP, DK, DV, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_fused_step, DK, DV, st, tk, s)
     DELTALOG_DISPATCH(desc, CALL_FUSED);
 #undef CALL_FUSED
     return DELTALOG_ERR_INVALID_ARG;
@@ -448,7 +461,7 @@ int deltalog_merge(const deltalog_desc *desc, const deltalog_state *state, const
     if (n == 0) return DELTALOG_OK;
     const StateArgs st = make_state_args(desc, state);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_MERGE(OP, D, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_merge, D, st, slot_idx, n, only_if_full, s)
+#define CALL_MERGE(OP, DK, DV, IO) DELTALOG_WITH_UL(OP, IO, desc, launch_merge, DK, DV, st, slot_idx, n, only_if_full, s)
     DELTALOG_DISPATCH(desc, CALL_MERGE);
 #undef CALL_MERGE
     return DELTALOG_ERR_INVALID_ARG;
@@ -463,13 +476,9 @@ int deltalog_reset_slots(const deltalog_desc *desc, const deltalog_state *state,
     const StateArgs st = make_state_args(desc, state);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool b16 = desc->base_dtype == DELTALOG_BF16;
-    if (desc->d_k == 64) {
-        if (b16) reset_slots_kernel<64, __nv_bfloat16><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
-        else reset_slots_kernel<64, float><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
-    } else {
-        if (b16) reset_slots_kernel<128, __nv_bfloat16><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
-        else reset_slots_kernel<128, float><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init);
-    }
+    const int tile = desc->d_k * desc->d_v;
+    if (b16) reset_slots_kernel<__nv_bfloat16><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init, tile);
+    else reset_slots_kernel<float><<<n * st.H, kThreads, 0, s>>>(st, slot_idx, S_init, tile);
     return finish_launch();
 }
 
@@ -482,7 +491,7 @@ int deltalog_eager_step(const deltalog_desc *desc, void *S, const void *q, const
     if (B == 0) return DELTALOG_OK;
     const TokenArgs tk = make_token_args(desc, q, k, v, g, beta, u_bonus, slot_idx, out, B);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-#define CALL_EAGER(OP, D, IO) return launch_eager<OP, D, IO>(S, desc, status, tk, s)
+#define CALL_EAGER(OP, DK, DV, IO) return launch_eager<OP, DK, DV, IO>(S, desc, status, tk, s)
     DELTALOG_DISPATCH(desc, CALL_EAGER);
 #undef CALL_EAGER
     return DELTALOG_ERR_INVALID_ARG;

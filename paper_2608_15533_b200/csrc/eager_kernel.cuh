@@ -11,14 +11,14 @@
 
 namespace deltalog {
 
-template <int OP, int D, typename IO, typename BT = float>
+template <int OP, int DK, int DV, typename IO, typename BT = float>
 __global__ void __launch_bounds__(kThreads, 2)
 eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *status, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
-    constexpr int DL = kVecDecay ? D : 1;
-    constexpr int C4 = D / 4, RL = kThreads / C4, NP = D / RL, EPL = D / 32;
+    constexpr int DL = kVecDecay ? DK : 1;
+    constexpr int C4 = DV / 4, RL = kThreads / C4, NP = DK / RL, EPL = DK / 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / H, h = blockIdx.x % H;
@@ -26,20 +26,20 @@ eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *s
     if (!resolve_slot(tk.slot_idx, b, num_slots, status, tid, slot)) return;
     const size_t unit = (size_t)slot * H + h, row = (size_t)b * H + h;
 
-    BT *Sg = static_cast<BT *>(S) + unit * D * D;
+    BT *Sg = static_cast<BT *>(S) + unit * DK * DV;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(p * RL + rl) * C4 + c4) * 4);
 
-    __shared__ __align__(16) float q_s[D], k_s[D], a_s[D], b_s[D];
-    __shared__ __align__(16) float red_s[2 * D * RL];
+    __shared__ __align__(16) float q_s[DK], k_s[DK], a_s[DK], b_s[DV];
+    __shared__ __align__(16) float red_s[2 * DV * RL];
     __shared__ float qk_s;
 
-    const IO *vg = static_cast<const IO *>(tk.v) + row * D;
-    if (tid < D) {
-        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * D + tid]);
-        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * D + tid]);
+    const IO *vg = static_cast<const IO *>(tk.v) + row * DV;
+    if (tid < DK) {
+        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * DK + tid]);
+        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * DK + tid]);
         a_s[tid] = tk.g ? expf(tk.g[row * DL + (kVecDecay ? tid : 0)]) : 1.f;  // no gate: plain linear attention
     }
     __syncthreads();
@@ -48,7 +48,7 @@ eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *s
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * DK + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -71,17 +71,17 @@ eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *s
     red4[(rl * 2 + 1) * C4 + c4] = aq;
     __syncthreads();
 
-    const int which = tid / D, c = tid % D;
-    const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+    const int which = tid / DV, c = tid % DV;
+    const bool active = kDelta ? (tid < 2 * DV) : (tid < DV);
     const int sel = kDelta ? which : 1;
     float y = 0.f;
     if (active) {
 #pragma unroll
-        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * DV + c];
     }
-    IO *og = static_cast<IO *>(tk.out) + row * D;
+    IO *og = static_cast<IO *>(tk.out) + row * DV;
     if (kDelta) {
-        if (tid < D) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
+        if (tid < DV) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
         __syncthreads();
         if (active && which == 1) og[c] = from_f32<IO>(scale * fmaf(qk_s, b_s[c], y));
     } else {

@@ -16,21 +16,22 @@
 
 namespace deltalog {
 
-template <int D>
+template <int DK, int DV>
 __host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
-    constexpr int RL = mat_threads<D>() / (D / 4);
-    // A [cap][D], U [cap][D], e, q, k, w, b [D] each, partial sums [RL][2][D], scalars
-    return sizeof(float) * ((size_t)2 * cap * D + 5 * D + 2 * D * RL + 4);
+    constexpr int RL = mat_threads<DK, DV>() / (DV / 4);
+    // A [cap][DK], U [cap][DV], e, q, k, w [DK] each, b [DV], partial sums [RL][2][DV], scalars
+    return sizeof(float) * ((size_t)cap * (DK + DV) + 4 * DK + DV + 2 * DV * RL + 4);
 }
 
-template <int OP, int D, typename IO, typename UL, typename BT = float>
-__global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
+template <int OP, int DK, int DV, typename IO, typename UL, typename BT = float>
+__global__ void __launch_bounds__(mat_threads<DK, DV>(), 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
-    constexpr int DL = kVecDecay ? D : 1;
-    constexpr int NT = mat_threads<D>();
-    constexpr int C4 = D / 4, RL = NT / C4, NP = D / RL, EPL = D / 32;
+    constexpr int DL = kVecDecay ? DK : 1;
+    constexpr int NT = mat_threads<DK, DV>();
+    constexpr int C4 = DV / 4, RL = NT / C4, NP = DK / RL, EPL = DK / 32;
+    static_assert(NT >= DK && NT >= (kDelta ? 2 : 1) * DV, "one thread per key channel and per output column");
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
@@ -39,7 +40,7 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
     const size_t unit = (size_t)slot * st.H + h, row = (size_t)b * st.H + h;
     const int cap = st.cap;
 
-    BT *Sg = static_cast<BT *>(st.S_base) + unit * D * D;
+    BT *Sg = static_cast<BT *>(st.S_base) + unit * DK * DV;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
@@ -49,18 +50,18 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
     len = len < 0 ? 0 : (len > cap ? cap : len);
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][D]  e^{lref_j - Lambda_ij} K_ij
-    float *U_s = A_s + (size_t)cap * D;                // [len][D]
-    float *e_s = U_s + (size_t)cap * D;                // e^{lref}
-    float *q_s = e_s + D;
-    float *k_s = q_s + D;
-    float *w_s = k_s + D;                              // RWKV6: e^{lambda_t}
-    float *b_s = w_s + D;
-    float *red_s = b_s + D;                            // [RL][2][D]
-    float *scal_s = red_s + 2 * D * RL;                // [0] = q.k  (or r.(bonus.k))
+    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][DK]  e^{lref_j - Lambda_ij} K_ij
+    float *U_s = A_s + (size_t)cap * DK;               // [len][DV]
+    float *e_s = U_s + (size_t)cap * DV;               // [DK] e^{lref}
+    float *q_s = e_s + DK;
+    float *k_s = q_s + DK;
+    float *w_s = k_s + DK;                             // RWKV6: e^{lambda_t}
+    float *b_s = w_s + DK;                             // [DV]
+    float *red_s = b_s + DV;                           // [RL][2][DV]
+    float *scal_s = red_s + 2 * DV * RL;               // [0] = q.k  (or r.(bonus.k))
 
-    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
-    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * DK;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * DV;
     const float *Lg = st.decay_log + unit * cap * DL;
     const float *lold = Lg + (size_t)(len > 0 ? len - 1 : 0) * DL;
     const float *gg = tk.g + row * DL;
@@ -68,28 +69,31 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
     // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
     if (!kVecDecay) {
         const float lref = (len > 0 ? lold[0] : 0.f) + (tk.g ? gg[0] : 0.f);  // no gate: plain linear attention
-        for (int x = tid * 4; x < len * D; x += NT * 4) {
-            const float wi = expf(lref - Lg[x / D]);
-            float kv[4], uv[4];
+        for (int x = tid * 4; x < len * DK; x += NT * 4) {
+            const float wi = expf(lref - Lg[x / DK]);
+            float kv[4];
             load_vec<IO, 4>(Kg + x, kv);
-            load_vec<UL, 4>(Ug + x, uv);
             *reinterpret_cast<float4 *>(A_s + x) = make_float4(wi * kv[0], wi * kv[1], wi * kv[2], wi * kv[3]);
+        }
+        for (int x = tid * 4; x < len * DV; x += NT * 4) {
+            float uv[4];
+            load_vec<UL, 4>(Ug + x, uv);
             *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
         }
     } else {
-        for (int x = tid; x < len * D; x += NT) {
-            const int i = x / D, j = x % D;
+        for (int x = tid; x < len * DK; x += NT) {
+            const int i = x / DK, j = x % DK;
             const float lref = lold[j] + (kPost ? gg[j] : 0.f);
-            A_s[x] = expf(lref - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);
-            U_s[x] = to_f32(Ug[x]);
+            A_s[x] = expf(lref - Lg[(size_t)i * DK + j]) * to_f32(Kg[x]);
         }
+        for (int x = tid; x < len * DV; x += NT) U_s[x] = to_f32(Ug[x]);
     }
-    const IO *vg = static_cast<const IO *>(tk.v) + row * D;
-    if (tid < D) {
+    const IO *vg = static_cast<const IO *>(tk.v) + row * DV;
+    if (tid < DK) {
         const int jl = kVecDecay ? tid : 0;
         const float lo = len > 0 ? lold[jl] : 0.f, lam = tk.g ? gg[jl] : 0.f;
-        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * D + tid]);
-        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * D + tid]);
+        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * DK + tid]);
+        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * DK + tid]);
         e_s[tid] = expf(kPost ? lo + lam : lo);
         w_s[tid] = expf(lam);
     }
@@ -100,7 +104,7 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * D + j];
+            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * DK + j];
             d = fmaf(q_s[j] * w, k_s[j], d);
         }
         d = warp_sum(d);
@@ -116,7 +120,7 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
     const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
     rank_update<NP>(
         s, len,
-        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP)[p4]; },
+        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * DK + rl * NP)[p4]; },
         [&](int i) { return U4[i * C4 + c4]; });
 
     // the two readouts from the materialised tile
@@ -132,17 +136,17 @@ __global__ void __launch_bounds__(mat_threads<D>(), 2) decode_merge_step_kernel(
     red4[(rl * 2 + 1) * C4 + c4] = aq;
     __syncthreads();
 
-    const int which = tid / D, c = tid % D;  // which: 0 -> S'^T k half, 1 -> S'^T q half
-    const bool active = kDelta ? (tid < 2 * D) : (tid < D);
+    const int which = tid / DV, c = tid % DV;  // which: 0 -> S'^T k half, 1 -> S'^T q half
+    const bool active = kDelta ? (tid < 2 * DV) : (tid < DV);
     const int sel = kDelta ? which : 1;
     float y = 0.f;
     if (active) {
 #pragma unroll
-        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * D + c];
+        for (int r = 0; r < RL; ++r) y += red_s[(r * 2 + sel) * DV + c];
     }
-    IO *og = static_cast<IO *>(tk.out) + row * D;
+    IO *og = static_cast<IO *>(tk.out) + row * DV;
     if (kDelta) {
-        if (tid < D) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
+        if (tid < DV) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
         __syncthreads();
         if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
     } else {

@@ -12,9 +12,9 @@
 
 namespace deltalog {
 
-template <int D>
+template <int DK, int DV>
 constexpr size_t merge_smem_bytes(int cap) {
-    return sizeof(float) * ((size_t)2 * cap * D + D);  // A [cap][D], U [cap][D] (fp32), e^{lbar} [D]
+    return sizeof(float) * ((size_t)cap * (DK + DV) + DK);  // A [cap][DK], U [cap][DV] (fp32), e^{lbar} [DK]
 }
 
 #ifndef DELTALOG_MERGE_PACK
@@ -28,13 +28,13 @@ constexpr int kMergePack = DELTALOG_MERGE_PACK;  // candidates per CTA of a pred
 // PACK: (listed slot, head) pairs a CTA is responsible for: 1 when every listed unit is expected to
 // fold, kMergePack (strided over the grid) for predicate merges over a batch with staggered fills, where most
 // pairs are skipped.
-template <int OP, int D, typename IO, typename UL, int PACK, typename BT = float>
-__global__ void __launch_bounds__(mat_threads<D>(), DELTALOG_MERGE_CTAS)
+template <int OP, int DK, int DV, typename IO, typename UL, int PACK, typename BT = float>
+__global__ void __launch_bounds__(mat_threads<DK, DV>(), DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
-    constexpr int DL = kVecDecay ? D : 1;
-    constexpr int NT = mat_threads<D>();
-    constexpr int C4 = D / 4, RL = NT / C4, NP = D / RL;
+    constexpr int DL = kVecDecay ? DK : 1;
+    constexpr int NT = mat_threads<DK, DV>();
+    constexpr int C4 = DV / 4, RL = NT / C4, NP = DK / RL;  // a thread owns NP consecutive rows x 4 columns
 
     const int tid = threadIdx.x;
     const int cap = st.cap;
@@ -78,39 +78,42 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     }
 
     // each thread owns rows [rl*NP, rl*NP + NP) x columns [4*c4, 4*c4 + 4)
-    BT *Sg = static_cast<BT *>(st.S_base) + unit * D * D;
+    BT *Sg = static_cast<BT *>(st.S_base) + unit * DK * DV;
     const int c4 = tid % C4, rl = tid / C4;
     float4 s[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4);
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][D]
-    float *U_s = A_s + (size_t)cap * D;                // [len][D]
-    float *e_s = U_s + (size_t)cap * D;                // [D]
+    float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][DK]
+    float *U_s = A_s + (size_t)cap * DK;               // [len][DV]
+    float *e_s = U_s + (size_t)cap * DV;               // [DK]
 
-    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * D;
-    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * D;
+    const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * DK;
+    const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * DV;
     const float *Lg = st.decay_log + unit * cap * DL;
     const float *lbar = Lg + (size_t)(len - 1) * DL;
     // key-side weights A_ij = e^{lbar_j - Lambda_ij} K_ij and the value-side rows
     if (!kVecDecay) {  // one weight per entry: four elements per thread and pass
-        for (int x = tid * 4; x < len * D; x += NT * 4) {
-            const float wi = expf(lbar[0] - Lg[x / D]);
-            float kv[4], uv[4];
+        for (int x = tid * 4; x < len * DK; x += NT * 4) {
+            const float wi = expf(lbar[0] - Lg[x / DK]);
+            float kv[4];
             load_vec<IO, 4>(Kg + x, kv);
-            load_vec<UL, 4>(Ug + x, uv);
             *reinterpret_cast<float4 *>(A_s + x) = make_float4(wi * kv[0], wi * kv[1], wi * kv[2], wi * kv[3]);
+        }
+        for (int x = tid * 4; x < len * DV; x += NT * 4) {
+            float uv[4];
+            load_vec<UL, 4>(Ug + x, uv);
             *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
         }
     } else {  // one weight per element (measured: the element-wise loop is the faster one here)
-        for (int x = tid; x < len * D; x += NT) {
-            const int i = x / D, j = x % D;
-            A_s[x] = expf(lbar[j] - Lg[(size_t)i * D + j]) * to_f32(Kg[x]);
-            U_s[x] = to_f32(Ug[x]);
+        for (int x = tid; x < len * DK; x += NT) {
+            const int i = x / DK, j = x % DK;
+            A_s[x] = expf(lbar[j] - Lg[(size_t)i * DK + j]) * to_f32(Kg[x]);
         }
+        for (int x = tid; x < len * DV; x += NT) U_s[x] = to_f32(Ug[x]);
     }
-    if (tid < D) e_s[tid] = expf(lbar[kVecDecay ? tid : 0]);
+    if (tid < DK) e_s[tid] = expf(lbar[kVecDecay ? tid : 0]);
     __syncthreads();
 
 #pragma unroll
@@ -121,7 +124,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     const float4 *U4 = reinterpret_cast<const float4 *>(U_s);
     rank_update<NP>(
         s, len,
-        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * D + rl * NP)[p4]; },
+        [&](int i, int p4) { return reinterpret_cast<const float4 *>(A_s + (size_t)i * DK + rl * NP)[p4]; },
         [&](int i) { return U4[i * C4 + c4]; });
 #pragma unroll
     for (int p = 0; p < NP; ++p) base_store4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4, s[p]);
@@ -130,16 +133,17 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
 }
 
 // Slot hand-over: empty the log of every head of the listed slots and, if given, install a new base.
-template <int D, typename BT = float>
-__global__ void __launch_bounds__(kThreads) reset_slots_kernel(StateArgs st, const int32_t *slot_idx, const float *S_init) {
+template <typename BT = float>
+__global__ void __launch_bounds__(kThreads) reset_slots_kernel(StateArgs st, const int32_t *slot_idx, const float *S_init,
+                                                               int tile_elems /* d_k * d_v */) {
     const int i = blockIdx.x / st.H, h = blockIdx.x % st.H;
     int slot;
     if (!resolve_slot(slot_idx, i, st.num_slots, st.status, threadIdx.x, slot)) return;
     const size_t unit = (size_t)slot * st.H + h;
     if (S_init) {
-        const float4 *src = reinterpret_cast<const float4 *>(S_init + ((size_t)i * st.H + h) * D * D);
-        BT *dst = static_cast<BT *>(st.S_base) + unit * D * D;
-        for (int x = threadIdx.x; x < D * D / 4; x += kThreads) base_store4<BT>(dst + 4 * x, src[x]);
+        const float4 *src = reinterpret_cast<const float4 *>(S_init + ((size_t)i * st.H + h) * tile_elems);
+        BT *dst = static_cast<BT *>(st.S_base) + unit * tile_elems;
+        for (int x = threadIdx.x; x < tile_elems / 4; x += kThreads) base_store4<BT>(dst + 4 * x, src[x]);
     }
     if (threadIdx.x == 0) st.log_len[unit] = 0;
 }

@@ -37,7 +37,7 @@ def make_desc(wl: Workload, cap: int, scale: float = 1.0):
     import paper_2608_15533_b200 as dl
 
     io = dl.F32 if wl.io_dtype == torch.float32 else dl.BF16
-    return dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.d, cap=cap, io_dtype=io, scale=scale)
+    return dl.Desc(op=wl.op, num_slots=wl.slots, H=wl.H, d_k=wl.d, d_v=wl.dv, cap=cap, io_dtype=io, scale=scale)
 
 
 @dataclass
@@ -165,7 +165,7 @@ def run_deltalog(wl: Workload, cap: int, device, *, units: Sequence[Tuple[int, i
             rows = step_slots if step_slots is not None else all_slots
             full = state.log_len[all_slots.long(), 0] == cap  # heads of a row fill in lockstep
             skip = torch.full_like(all_slots, -1)
-            out = torch.zeros(wl.batch, wl.H, wl.d, dtype=wl.io_dtype, device=device)
+            out = torch.zeros(wl.batch, wl.H, wl.dv, dtype=wl.io_dtype, device=device)
             for fn, sel in ((dl.decode_step, ~full), (dl.decode_merge_step, full)):
                 if bool(sel.any()):
                     fn(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,

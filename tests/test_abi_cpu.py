@@ -56,7 +56,8 @@ def test_host_side_rejections_launch_nothing(lib):
     s = _state()
     assert _decode(lib, _desc(op=7), s) == binding.ERR_INVALID_ARG
     assert _decode(lib, _desc(d_k=96, d_v=96), s) == binding.ERR_UNSUPPORTED_SHAPE
-    assert _decode(lib, _desc(d_k=64, d_v=128), s) == binding.ERR_UNSUPPORTED_SHAPE
+    assert _decode(lib, _desc(d_k=64, d_v=96), s) == binding.ERR_UNSUPPORTED_SHAPE
+    assert _decode(lib, _desc(d_k=256, d_v=128), s) == binding.ERR_UNSUPPORTED_SHAPE
     assert _decode(lib, _desc(cap=0), s) == binding.ERR_CAP_RANGE
     assert _decode(lib, _desc(cap=65), s) == binding.ERR_CAP_RANGE
     # a 16-bit U log for the delta rule needs 16-bit I/O; where b = v the U log has the I/O dtype

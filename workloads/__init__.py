@@ -36,7 +36,7 @@ class Workload:
     op: int
     batch: int            # sequences decoded per step
     H: int
-    d: int                # d_k == d_v
+    d: int                # key dimension d_k (and d_v unless ``d_v`` is given)
     steps: int
     caps: Tuple[int, ...]  # log capacities exercised
     io_dtype: torch.dtype = torch.bfloat16
@@ -44,6 +44,11 @@ class Workload:
     num_slots: Optional[int] = None   # state-pool size (>= batch); None -> batch
     staggered: bool = False           # random initial log fill per sequence
     seed: int = 0
+    d_v: Optional[int] = None         # value dimension when it differs from the key dimension
+
+    @property
+    def dv(self) -> int:
+        return self.d if self.d_v is None else self.d_v
 
     @property
     def slots(self) -> int:
@@ -99,7 +104,7 @@ class TokenSource:
         assert not self._drew_state, "initial_state() is the first draw"
         self._drew_state = True
         wl = self.wl
-        return self._randn(wl.slots, wl.H, wl.d, wl.d).mul_(0.1)
+        return self._randn(wl.slots, wl.H, wl.d, wl.dv).mul_(0.1)
 
     def bonus(self) -> Optional[torch.Tensor]:
         """RWKV6 bonus ``[H, d] ~ N(0, 0.1^2)`` fp32 (drawn right after the state); None otherwise."""
@@ -111,7 +116,7 @@ class TokenSource:
         """One token batch: ``q, k, v [B,H,d]`` in the I/O dtype, ``g`` fp32 log-decay, ``beta`` fp32."""
         wl = self.wl
         B, H, d = wl.batch, wl.H, wl.d
-        q, k, v = self._randn(B, H, d), self._randn(B, H, d), self._randn(B, H, d)
+        q, k, v = self._randn(B, H, d), self._randn(B, H, d), self._randn(B, H, wl.dv)
         if wl.op == RWKV6:
             g = -torch.exp(self._randn(B, H, d).mul_(0.5).sub_(0.5))
             _ = self._randn(B, H)  # keeps the draw order uniform across operators
