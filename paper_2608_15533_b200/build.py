@@ -17,6 +17,7 @@ NVCC_FLAGS = [
     "-O3", "-std=c++17", "-lineinfo",
     "--shared", "-Xcompiler", "-fPIC",
     "-Xptxas", "-v",
+    "--threads", "0",   # the translation units under csrc/ compile side by side
 ]
 
 

@@ -155,7 +155,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 // Wait for a phase of an mbarrier, giving up after kWaitLimitNs or as soon as the CTA aborts.
 // (The polling loop is kept out of line: the kernel's roles share the SM's instruction caches, and a
 // dozen inlined copies of it were a measurable part of the instruction-fetch traffic.)
-__device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+static __device__ __noinline__ bool bounded_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     const unsigned long long t0 = global_timer_ns();
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
