@@ -16,9 +16,12 @@ constexpr int kWarps = kThreads / 32;
 #ifndef DELTALOG_MAT_THREADS
 #define DELTALOG_MAT_THREADS 256
 #endif
+#ifndef DELTALOG_MAT_THREADS_64
+#define DELTALOG_MAT_THREADS_64 128
+#endif
 template <int DK, int DV>
 __host__ __device__ constexpr int mat_threads() {
-    return (DK >= 128 && DV >= 128) ? DELTALOG_MAT_THREADS : 256;
+    return (DK >= 128 && DV >= 128) ? DELTALOG_MAT_THREADS : (DK * DV <= 64 * 64 ? DELTALOG_MAT_THREADS_64 : 256);
 }
 constexpr int kMaxCap = 64;
 

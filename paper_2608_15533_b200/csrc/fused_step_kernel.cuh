@@ -16,15 +16,18 @@
 
 namespace deltalog {
 
-template <int DK, int DV>
-__host__ __device__ constexpr size_t fused_step_smem_bytes(int cap) {
+template <int DK, int DV, typename IO, typename UL>
+__host__ __device__ constexpr size_t fused_step_smem_bytes(int cap, bool vec_decay) {
     constexpr int RL = mat_threads<DK, DV>() / (DV / 4);
-    // A [cap][DK], U [cap][DV], e, q, k, w [DK] each, b [DV], partial sums [RL][2][DV], scalars
-    return sizeof(float) * ((size_t)cap * (DK + DV) + 4 * DK + DV + 2 * DV * RL + 4);
+    // A [cap][DK], U [cap][DV], e, q, k, w [DK] each, b [DV], partial sums [RL][2][DV], scalars; then the log as
+    // it is stored (requested ahead of the length word): K [cap][DK], Lambda [cap][d_lambda], U where not fp32
+    return sizeof(float) * ((size_t)cap * (DK + DV) + 4 * DK + DV + 2 * DV * RL + 4) + sizeof(IO) * (size_t)cap * DK +
+           sizeof(float) * (((size_t)cap * (vec_decay ? DK : 1) + 3) / 4 * 4) +
+           (sizeof(UL) == 4 ? 0 : sizeof(UL) * (size_t)cap * DV);
 }
 
 template <int OP, int DK, int DV, typename IO, typename UL, typename BT = float>
-__global__ void __launch_bounds__(mat_threads<DK, DV>(), 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
+__global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <= 128 ? 4 : 2) decode_merge_step_kernel(StateArgs st, TokenArgs tk) {
     constexpr bool kDelta = OpTraits<OP>::kDeltaRule;
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
@@ -46,9 +49,6 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), 2) decode_merge_step_ke
 #pragma unroll
     for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4);
 
-    int len = st.log_len[unit];
-    len = len < 0 ? 0 : (len > cap ? cap : len);
-
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][DK]  e^{lref_j - Lambda_ij} K_ij
     float *U_s = A_s + (size_t)cap * DK;               // [len][DV]
@@ -59,12 +59,55 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), 2) decode_merge_step_ke
     float *b_s = w_s + DK;                             // [DV]
     float *red_s = b_s + DV;                           // [RL][2][DV]
     float *scal_s = red_s + 2 * DV * RL;               // [0] = q.k  (or r.(bonus.k))
+    IO *K_raw = reinterpret_cast<IO *>(scal_s + 4);    // [cap][DK] as stored
+    float *L_raw = reinterpret_cast<float *>(K_raw + (size_t)cap * DK);  // [cap][DL]
+    UL *U_raw = sizeof(UL) == 4 ? reinterpret_cast<UL *>(U_s) : reinterpret_cast<UL *>(L_raw + ((size_t)cap * DL + 3) / 4 * 4);
 
     const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * DK;
     const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * DV;
     const float *Lg = st.decay_log + unit * cap * DL;
-    const float *lold = Lg + (size_t)(len > 0 ? len - 1 : 0) * DL;
+    // The whole log is requested (asynchronously, into shared memory) together with the tile, BEFORE the length
+    // word is known: a CTA's run time is one chain of dependent memory round trips, and this takes one of them
+    // out.  Entries beyond the live length are never used.  (Needs 16-byte aligned snapshot rows.)
+    const bool ahead = kVecDecay || cap % 4 == 0;
+    if (ahead) {
+        cta_cp_async(K_raw, Kg, cap * DK * (int)sizeof(IO), tid, NT);
+        cta_cp_async(U_raw, Ug, cap * DV * (int)sizeof(UL), tid, NT);
+        cta_cp_async(L_raw, Lg, (cap * DL * 4 + 15) / 16 * 16, tid, NT);
+        cp_async_commit();
+    }
+    int len = st.log_len[unit];
+    len = len < 0 ? 0 : (len > cap ? cap : len);
+    const float *lold = (ahead ? L_raw : Lg) + (size_t)(len > 0 ? len - 1 : 0) * DL;
     const float *gg = tk.g + row * DL;
+    if (ahead) {
+        cp_async_wait_all();
+        __syncthreads();
+        for (int x = tid * 4; x < len * DK; x += NT * 4) {
+            const int i = x / DK, j = x % DK;
+            float kv[4], w[4];
+            load_vec<IO, 4>(K_raw + x, kv);
+            if (kVecDecay) {
+                const float4 lo = *reinterpret_cast<const float4 *>(lold + j);
+                const float4 li = *reinterpret_cast<const float4 *>(L_raw + (size_t)i * DK + j);
+                float4 gl = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (kPost) gl = *reinterpret_cast<const float4 *>(gg + j);
+                w[0] = expf(lo.x + gl.x - li.x), w[1] = expf(lo.y + gl.y - li.y);
+                w[2] = expf(lo.z + gl.z - li.z), w[3] = expf(lo.w + gl.w - li.w);
+            } else {
+                const float lref = lold[0] + (tk.g ? gg[0] : 0.f);  // (len > 0 here) no gate: plain linear attention
+                w[0] = w[1] = w[2] = w[3] = expf(lref - L_raw[i]);
+            }
+            *reinterpret_cast<float4 *>(A_s + x) = make_float4(w[0] * kv[0], w[1] * kv[1], w[2] * kv[2], w[3] * kv[3]);
+        }
+        if (sizeof(UL) != 4) {
+            for (int x = tid * 4; x < len * DV; x += NT * 4) {
+                float uv[4];
+                load_vec<UL, 4>(U_raw + x, uv);
+                *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
+            }
+        }
+    } else
     // lref: the decay level the state is materialised at -- lbar' for the delta rule (both readouts
     // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
     if (!kVecDecay) {

@@ -8,7 +8,7 @@ namespace {
 template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
     auto kernel = decode_merge_step_kernel<OP, DK, DV, IO, UL, BT>;
-    const size_t smem = fused_step_smem_bytes<DK, DV>(st.cap);
+    const size_t smem = fused_step_smem_bytes<DK, DV, IO, UL>(st.cap, OpTraits<OP>::kVecDecay);
     if (int rc = ensure_smem(kernel, smem)) return rc;
     kernel<<<tk.B * st.H, mat_threads<DK, DV>(), smem, stream>>>(st, tk);
     return finish_launch();

@@ -25,7 +25,7 @@ int launch_merge(const StateArgs &st, const int32_t *slot_idx, int32_t n, int32_
             return finish_launch();
         }
     }
-    const size_t smem = merge_smem_bytes<DK, DV>(st.cap);
+    const size_t smem = merge_smem_bytes<DK, DV, IO, UL>(st.cap, OpTraits<OP>::kVecDecay);
     // Without the predicate every listed unit is expected to fold: one unit per CTA.  With it (one
     // call over a whole batch whose fills are staggered) most units are skipped: kMergePack candidates per CTA.
     const int pairs = n * st.H;

@@ -12,9 +12,13 @@
 
 namespace deltalog {
 
-template <int DK, int DV>
-constexpr size_t merge_smem_bytes(int cap) {
-    return sizeof(float) * ((size_t)cap * (DK + DV) + DK);  // A [cap][DK], U [cap][DV] (fp32), e^{lbar} [DK]
+// A [cap][DK], U [cap][DV] (fp32), e^{lbar} [DK]; then the log as it is stored, requested ahead of the length
+// word: K [cap][DK] (I/O dtype), Lambda [cap][d_lambda] (fp32), and U [cap][DV] where it is not fp32 already.
+template <int DK, int DV, typename IO, typename UL>
+constexpr size_t merge_smem_bytes(int cap, bool vec_decay) {
+    return sizeof(float) * ((size_t)cap * (DK + DV) + DK) + sizeof(IO) * (size_t)cap * DK +
+           sizeof(float) * (((size_t)cap * (vec_decay ? DK : 1) + 3) / 4 * 4) +
+           (sizeof(UL) == 4 ? 0 : sizeof(UL) * (size_t)cap * DV);
 }
 
 #ifndef DELTALOG_MERGE_PACK
@@ -29,7 +33,7 @@ constexpr int kMergePack = DELTALOG_MERGE_PACK;  // candidates per CTA of a pred
 // fold, kMergePack (strided over the grid) for predicate merges over a batch with staggered fills, where most
 // pairs are skipped.
 template <int OP, int DK, int DV, typename IO, typename UL, int PACK, typename BT = float>
-__global__ void __launch_bounds__(mat_threads<DK, DV>(), DELTALOG_MERGE_CTAS)
+__global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <= 128 ? 2 * DELTALOG_MERGE_CTAS : DELTALOG_MERGE_CTAS)
 merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_t n_pairs) {
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? DK : 1;
@@ -73,8 +77,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
         int slot;
         if (!resolve_slot(slot_idx, pair / st.H, st.num_slots, st.status, tid, slot)) return;
         unit = (size_t)slot * st.H + pair % st.H;
-        len = st.log_len[unit];
-        if (len <= 0 || len > cap || (only_if_full && len < cap)) return;  // nothing to fold: no dense write
+        len = 0;  // read below, after the tile and the log have been requested
     }
 
     // each thread owns rows [rl*NP, rl*NP + NP) x columns [4*c4, 4*c4 + 4)
@@ -88,10 +91,57 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
     float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][DK]
     float *U_s = A_s + (size_t)cap * DK;               // [len][DV]
     float *e_s = U_s + (size_t)cap * DV;               // [DK]
+    IO *K_raw = reinterpret_cast<IO *>(e_s + DK);      // [cap][DK] as stored
+    float *L_raw = reinterpret_cast<float *>(K_raw + (size_t)cap * DK);  // [cap][DL]
+    UL *U_raw = sizeof(UL) == 4 ? reinterpret_cast<UL *>(U_s) : reinterpret_cast<UL *>(L_raw + ((size_t)cap * DL + 3) / 4 * 4);
 
     const IO *Kg = static_cast<const IO *>(st.K_log) + unit * cap * DK;
     const UL *Ug = static_cast<const UL *>(st.U_log) + unit * cap * DV;
     const float *Lg = st.decay_log + unit * cap * DL;
+    // Without the predicate every listed unit is expected to hold a full log: the whole log is requested
+    // (asynchronously, into shared memory) together with the tile, BEFORE the length word is known -- a CTA's
+    // run time is one chain of dependent memory round trips, and this takes one of them out.  Entries beyond
+    // the live length are never used.  (Needs 16-byte aligned snapshot rows: cap % 4 == 0 for scalar decay.)
+    const bool ahead = PACK == 1 && (kVecDecay || cap % 4 == 0);
+    if (ahead) {
+        cta_cp_async(K_raw, Kg, cap * DK * (int)sizeof(IO), tid, NT);
+        cta_cp_async(U_raw, Ug, cap * DV * (int)sizeof(UL), tid, NT);
+        cta_cp_async(L_raw, Lg, (cap * DL * 4 + 15) / 16 * 16, tid, NT);
+        cp_async_commit();
+    }
+    if (PACK == 1) {
+        len = st.log_len[unit];
+        if (len <= 0 || len > cap || (only_if_full && len < cap)) {  // nothing to fold: no dense write
+            cp_async_wait_all();
+            return;
+        }
+    }
+    if (ahead) {
+        cp_async_wait_all();
+        __syncthreads();
+        const float *lbar_s = L_raw + (size_t)(len - 1) * DL;
+        for (int x = tid * 4; x < len * DK; x += NT * 4) {
+            const int i = x / DK, j = x % DK;
+            float kv[4], w[4];
+            load_vec<IO, 4>(K_raw + x, kv);
+            if (kVecDecay) {
+                const float4 lb = *reinterpret_cast<const float4 *>(lbar_s + j);
+                const float4 li = *reinterpret_cast<const float4 *>(L_raw + (size_t)i * DK + j);
+                w[0] = expf(lb.x - li.x), w[1] = expf(lb.y - li.y), w[2] = expf(lb.z - li.z), w[3] = expf(lb.w - li.w);
+            } else {
+                w[0] = w[1] = w[2] = w[3] = expf(lbar_s[0] - L_raw[i]);
+            }
+            *reinterpret_cast<float4 *>(A_s + x) = make_float4(w[0] * kv[0], w[1] * kv[1], w[2] * kv[2], w[3] * kv[3]);
+        }
+        if (sizeof(UL) != 4) {
+            for (int x = tid * 4; x < len * DV; x += NT * 4) {
+                float uv[4];
+                load_vec<UL, 4>(U_raw + x, uv);
+                *reinterpret_cast<float4 *>(U_s + x) = make_float4(uv[0], uv[1], uv[2], uv[3]);
+            }
+        }
+        if (tid < DK) e_s[tid] = expf(lbar_s[kVecDecay ? tid : 0]);
+    } else {
     const float *lbar = Lg + (size_t)(len - 1) * DL;
     // key-side weights A_ij = e^{lbar_j - Lambda_ij} K_ij and the value-side rows
     if (!kVecDecay) {  // one weight per entry: four elements per thread and pass
@@ -114,6 +164,7 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
         for (int x = tid; x < len * DV; x += NT) U_s[x] = to_f32(Ug[x]);
     }
     if (tid < DK) e_s[tid] = expf(lbar[kVecDecay ? tid : 0]);
+    }
     __syncthreads();
 
 #pragma unroll
