@@ -37,14 +37,17 @@ ADDITIVE = (LINATTN, RETNET, GLA)  # b = v, readout from the updated state; LINA
 class LogState:
     """Base + bounded log for ``N`` independent (sequence, head) units (Section 3.1)."""
 
-    def __init__(self, op: int, S0: np.ndarray, cap: int, store_u=None, store_base=None):
+    def __init__(self, op: int, S0: np.ndarray, cap: int, store_u=None, store_base=None, store_lam=None):
         """``store_u``: optional function applied to a value-side factor when it is written into the
         log (e.g. rounding to a 16-bit format), for studies of reduced-precision logs; None = exact.
         ``store_base``: the same for every write of the dense base (the initial state, Eq. 5) -- the
-        base is then only re-rounded once per materialisation, not once per token."""
+        base is then only re-rounded once per materialisation, not once per token.
+        ``store_lam``: the same for every log-decay snapshot written into the log (the running
+        cumulative log-decay ``lbar`` itself stays exact), for studies of more compact snapshots."""
         S0 = np.asarray(S0, dtype=np.float64)
         self.store_u = store_u
         self.store_base = store_base
+        self.store_lam = store_lam
         self.op = int(op)
         self.N, self.d_k, self.d_v = S0.shape
         self.cap = int(cap)
@@ -120,7 +123,7 @@ def decode_step(st: LogState, q, k, v, lam, beta=None, bonus=None, scale: float 
         # lines 4-5 / Eq. 4: append (a, b, lbar) into slot L; the base is untouched
         st.K_log[n, L] = a
         st.U_log[n, L] = b if st.store_u is None else st.store_u(b)
-        st.Lam_log[n, L] = st.lbar[n]
+        st.Lam_log[n, L] = st.lbar[n] if st.store_lam is None else st.store_lam(st.lbar[n])
         st.length[n] = L + 1
         if st.op != RWKV6:
             S_new = materialize_unit(st.S_base[n], st.lbar[n], st.K_log[n], st.U_log[n], st.Lam_log[n], L + 1)
