@@ -103,6 +103,9 @@ def main(argv=None):
     ap.add_argument("--command", required=True, help="the full ncu command line that produced the CSV")
     ap.add_argument("--build-id", default=None, help="identifier of the profiled build (default: the current sources)")
     ap.add_argument("--out", type=Path, default=DEFAULT_OUT)
+    ap.add_argument("--add", action="store_true",
+                    help="add the kernel families of this capture to the configuration's record instead of replacing it "
+                         "(a second command of the same configuration, e.g. the eager kernel or the paper's cycle)")
     args = ap.parse_args(argv)
 
     build_id = args.build_id or build.source_id(build.extra_flags())
@@ -114,7 +117,13 @@ def main(argv=None):
         doc = {"build_id": build_id, "captures": {}}
     doc["what"] = ("dram__bytes_read.sum / dram__bytes_write.sum per launch (mean over the captured launches), "
                    "ncu --cache-control none: L2 as the previous launch of the loop left it")
-    doc["captures"][capture_key(args.config, args.cap, args.state)] = {"command": args.command, "kernels": kernels}
+    key = capture_key(args.config, args.cap, args.state)
+    if args.add and key in doc["captures"]:
+        rec = doc["captures"][key]
+        rec["kernels"].update(kernels)
+        rec.setdefault("more_commands", []).append(args.command)
+    else:
+        doc["captures"][key] = {"command": args.command, "kernels": kernels}
     args.out.write_text(json.dumps(doc, indent=1, sort_keys=True) + "\n")
     for fam, k in kernels.items():
         print(f"{fam:8s} {k['launches']:3d} launches  read {k['dram_read_bytes_per_launch'] / 1e6:8.1f} MB  "
