@@ -19,9 +19,9 @@ namespace deltalog {
 template <int DK, int DV, typename IO, typename UL>
 __host__ __device__ constexpr size_t fused_step_smem_bytes(int cap, bool vec_decay) {
     constexpr int RL = mat_threads<DK, DV>() / (DV / 4);
-    // A [cap][DK], U [cap][DV], e, q, k, w [DK] each, b [DV], partial sums [RL][2][DV], scalars; then the log as
+    // A [cap][DK], U [cap][DV], e, q, k, w, lambda [DK] each, b [DV], partial sums [RL][2][DV], scalars; then the log as
     // it is stored (requested ahead of the length word): K [cap][DK], Lambda [cap][d_lambda], U where not fp32
-    return sizeof(float) * ((size_t)cap * (DK + DV) + 4 * DK + DV + 2 * DV * RL + 4) + sizeof(IO) * (size_t)cap * DK +
+    return sizeof(float) * ((size_t)cap * (DK + DV) + 5 * DK + DV + 2 * DV * RL + 4) + sizeof(IO) * (size_t)cap * DK +
            sizeof(float) * (((size_t)cap * (vec_decay ? DK : 1) + 3) / 4 * 4) +
            (sizeof(UL) == 4 ? 0 : sizeof(UL) * (size_t)cap * DV);
 }
@@ -48,6 +48,21 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     float4 s[NP];
 #pragma unroll
     for (int p = 0; p < NP; ++p) s[p] = base_load4<BT>(Sg + ((size_t)(rl * NP + p) * C4 + c4) * 4);
+    // The token's vectors are requested here as well, into registers: nothing below waits for global memory
+    // a second time (a CTA's run time is one chain of dependent round trips).
+    const float *gg = tk.g + row * (kVecDecay ? DK : 1);
+    const IO *vg = static_cast<const IO *>(tk.v) + row * DV;
+    // (Measured on the same box: GDN shape 123 -> 113 us, RWKV6 shape unchanged, KDA shape 252 -> 262 us.)
+    float q_r = 0.f, k_r = 0.f, lam_r = 0.f, v_r = 0.f, beta_r = 0.f, bonus_r[EPL];
+    if (tid < DK) {
+        q_r = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * DK + tid]);
+        k_r = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * DK + tid]);
+    }
+    if (tid < DK || !kVecDecay) lam_r = tk.g ? gg[kVecDecay ? tid : 0] : 0.f;  // no gate: plain linear attention
+    if (tid < DV) v_r = to_f32(vg[tid]);
+    if (kDelta) beta_r = tk.beta[row];
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) bonus_r[e] = (!kPost && warp == 0) ? tk.u_bonus[(size_t)h * DK + lane + 32 * e] : 1.f;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float *A_s = reinterpret_cast<float *>(smem_raw);  // [len][DK]  e^{lref_j - Lambda_ij} K_ij
@@ -59,7 +74,8 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     float *b_s = w_s + DK;                             // [DV]
     float *red_s = b_s + DV;                           // [RL][2][DV]
     float *scal_s = red_s + 2 * DV * RL;               // [0] = q.k  (or r.(bonus.k))
-    IO *K_raw = reinterpret_cast<IO *>(scal_s + 4);    // [cap][DK] as stored
+    float *lam_s = scal_s + 4;                         // [DK] the token's log-decay
+    IO *K_raw = reinterpret_cast<IO *>(lam_s + DK);    // [cap][DK] as stored
     float *L_raw = reinterpret_cast<float *>(K_raw + (size_t)cap * DK);  // [cap][DL]
     UL *U_raw = sizeof(UL) == 4 ? reinterpret_cast<UL *>(U_s) : reinterpret_cast<UL *>(L_raw + ((size_t)cap * DL + 3) / 4 * 4);
 
@@ -79,7 +95,7 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     int len = st.log_len[unit];
     len = len < 0 ? 0 : (len > cap ? cap : len);
     const float *lold = (ahead ? L_raw : Lg) + (size_t)(len > 0 ? len - 1 : 0) * DL;
-    const float *gg = tk.g + row * DL;
+    if (tid < DK) lam_s[tid] = lam_r;   // the token's log-decay per key channel, for the weights below
     if (ahead) {
         cp_async_wait_all();
         __syncthreads();
@@ -91,11 +107,11 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
                 const float4 lo = *reinterpret_cast<const float4 *>(lold + j);
                 const float4 li = *reinterpret_cast<const float4 *>(L_raw + (size_t)i * DK + j);
                 float4 gl = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (kPost) gl = *reinterpret_cast<const float4 *>(gg + j);
+                if (kPost) gl = *reinterpret_cast<const float4 *>(lam_s + j);
                 w[0] = expf(lo.x + gl.x - li.x), w[1] = expf(lo.y + gl.y - li.y);
                 w[2] = expf(lo.z + gl.z - li.z), w[3] = expf(lo.w + gl.w - li.w);
             } else {
-                const float lref = lold[0] + (tk.g ? gg[0] : 0.f);  // (len > 0 here) no gate: plain linear attention
+                const float lref = lold[0] + lam_s[0];  // (len > 0 here)
                 w[0] = w[1] = w[2] = w[3] = expf(lref - L_raw[i]);
             }
             *reinterpret_cast<float4 *>(A_s + x) = make_float4(w[0] * kv[0], w[1] * kv[1], w[2] * kv[2], w[3] * kv[3]);
@@ -111,7 +127,7 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     // lref: the decay level the state is materialised at -- lbar' for the delta rule (both readouts
     // are taken on the decayed state), lbar for RWKV6 (readout on the pre-update state).
     if (!kVecDecay) {
-        const float lref = (len > 0 ? lold[0] : 0.f) + (tk.g ? gg[0] : 0.f);  // no gate: plain linear attention
+        const float lref = (len > 0 ? lold[0] : 0.f) + lam_r;  // (scalar decay: every thread below DK holds it)
         for (int x = tid * 4; x < len * DK; x += NT * 4) {
             const float wi = expf(lref - Lg[x / DK]);
             float kv[4];
@@ -131,14 +147,13 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
         }
         for (int x = tid; x < len * DV; x += NT) U_s[x] = to_f32(Ug[x]);
     }
-    const IO *vg = static_cast<const IO *>(tk.v) + row * DV;
     if (tid < DK) {
         const int jl = kVecDecay ? tid : 0;
-        const float lo = len > 0 ? lold[jl] : 0.f, lam = tk.g ? gg[jl] : 0.f;
-        q_s[tid] = to_f32(static_cast<const IO *>(tk.q)[tk.qk_row(b, h) * DK + tid]);
-        k_s[tid] = to_f32(static_cast<const IO *>(tk.k)[tk.qk_row(b, h) * DK + tid]);
-        e_s[tid] = expf(kPost ? lo + lam : lo);
-        w_s[tid] = expf(lam);
+        const float lo = len > 0 ? lold[jl] : 0.f;
+        q_s[tid] = q_r;
+        k_s[tid] = k_r;
+        e_s[tid] = expf(kPost ? lo + lam_r : lo);
+        w_s[tid] = expf(lam_r);
     }
     __syncthreads();
 
@@ -147,8 +162,7 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
 #pragma unroll
         for (int e = 0; e < EPL; ++e) {
             const int j = lane + 32 * e;
-            const float w = kPost ? 1.f : tk.u_bonus[(size_t)h * DK + j];
-            d = fmaf(q_s[j] * w, k_s[j], d);
+            d = fmaf(q_s[j] * bonus_r[e], k_s[j], d);
         }
         d = warp_sum(d);
         if (lane == 0) scal_s[0] = d;
@@ -189,12 +203,12 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     }
     IO *og = static_cast<IO *>(tk.out) + row * DV;
     if (kDelta) {
-        if (tid < DV) b_s[c] = tk.beta[row] * (to_f32(vg[c]) - y);
+        if (tid < DV) b_s[c] = beta_r * (v_r - y);
         __syncthreads();
         if (active && which == 1) og[c] = from_f32<IO>(st.scale * fmaf(scal_s[0], b_s[c], y));
     } else {
         if (active) {
-            const float vv = to_f32(vg[c]);
+            const float vv = v_r;   // (active threads are the first DV: c == tid)
             b_s[c] = vv;
             og[c] = from_f32<IO>((kPost ? st.scale : 1.f) * fmaf(scal_s[0], vv, y));
         }
