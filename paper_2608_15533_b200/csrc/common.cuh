@@ -73,6 +73,19 @@ __device__ __forceinline__ void load_vec<__nv_bfloat16, 2>(const __nv_bfloat16 *
     out[0] = __uint_as_float(v << 16), out[1] = __uint_as_float(v & 0xffff0000u);
 }
 
+// Eight consecutive elements as 16-byte accesses, widened to fp32.
+__device__ __forceinline__ void load8(const float *p, float (&out)[8]) {
+    const float4 a = reinterpret_cast<const float4 *>(p)[0], b = reinterpret_cast<const float4 *>(p)[1];
+    out[0] = a.x, out[1] = a.y, out[2] = a.z, out[3] = a.w, out[4] = b.x, out[5] = b.y, out[6] = b.z, out[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16 *p, float (&out)[8]) {
+    const uint4 v = *reinterpret_cast<const uint4 *>(p);
+    out[0] = __uint_as_float(v.x << 16), out[1] = __uint_as_float(v.x & 0xffff0000u);
+    out[2] = __uint_as_float(v.y << 16), out[3] = __uint_as_float(v.y & 0xffff0000u);
+    out[4] = __uint_as_float(v.z << 16), out[5] = __uint_as_float(v.z & 0xffff0000u);
+    out[6] = __uint_as_float(v.w << 16), out[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+
 #ifndef DELTALOG_STREAM_BASE
 #define DELTALOG_STREAM_BASE 1
 #endif

@@ -625,55 +625,53 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
                     group_sync(1);
                     if (gtid == 0) mbar_arrive(prep_done + 8u * (j & (NS - 1)));  // the stream group may start on this unit
 
-                    // key-side replay coefficients: each lane owns EPL consecutive key channels; a warp
-                    // takes entries gwarp, gwarp+4, ... two at a time so that their reductions overlap
-                    float qv[EPL], kv[EPL], lb[EPL];
-                    load_vec<float, EPL>(q_s + lane * EPL, qv);
-                    load_vec<float, EPL>(k_s + lane * EPL, kv);
-                    if (kVecDecay) load_vec<float, EPL>(lbar_s + lane * EPL, lb);
-                    for (int i0 = gwarp; i0 < len; i0 += 2 * kHalf) {
-                        const int i1 = i0 + kHalf;
-                        const bool two = i1 < len;
-                        float dq0 = 0.f, dk0 = 0.f, dq1 = 0.f, dk1 = 0.f;
-                        float ke[EPL], le[EPL];
-                        load_vec<IO, EPL>(K_a + i0 * D + lane * EPL, ke);
-                        if (kVecDecay) load_vec<float, EPL>(L_a + i0 * D + lane * EPL, le);
+                    // Key-side replay coefficients, sixteen entries per round of the group: eight lanes share an
+                    // entry (a lane takes 2 x 8 key channels with 16-byte loads), a warp pass covers four entries
+                    // and the sums are combined in three shuffle rounds.  (With a whole warp per entry -- eight
+                    // entries per round, five shuffle rounds -- the launch time climbed in steps at 9, 17, 25 live
+                    // entries: from the second round on this group was the slowest stage.)
+                    {
+                        const int s8 = lane & 7, e4 = lane >> 3;
+                        for (int i0 = 4 * gwarp; i0 < len; i0 += 4 * kHalf) {
+                            const int i = i0 + e4;
+                            float dq = 0.f, dk = 0.f;
+                            if (i < len) {
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) {
-                            const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
-                            dq0 = fmaf(qv[e], kij, dq0);
-                            if (kDelta) dk0 = fmaf(kv[e], kij, dk0);
-                        }
-                        if (two) {
-                            load_vec<IO, EPL>(K_a + i1 * D + lane * EPL, ke);
-                            if (kVecDecay) load_vec<float, EPL>(L_a + i1 * D + lane * EPL, le);
+                                for (int hh = 0; hh < D / 64; ++hh) {
+                                    const int ch = 8 * s8 + 64 * hh;
+                                    float q8[8], k8[8], ke[8];
+                                    load8(q_s + ch, q8);
+                                    if (kDelta) load8(k_s + ch, k8);
+                                    load8(K_a + i * D + ch, ke);
+                                    if (kVecDecay) {
+                                        float lb8[8], le[8];
+                                        load8(lbar_s + ch, lb8);
+                                        load8(L_a + i * D + ch, le);
 #pragma unroll
-                            for (int e = 0; e < EPL; ++e) {
-                                const float kij = kVecDecay ? ke[e] * expf(lb[e] - le[e]) : ke[e];
-                                dq1 = fmaf(qv[e], kij, dq1);
-                                if (kDelta) dk1 = fmaf(kv[e], kij, dk1);
+                                        for (int e = 0; e < 8; ++e) ke[e] *= expf(lb8[e] - le[e]);
+                                    }
+#pragma unroll
+                                    for (int e = 0; e < 8; ++e) {
+                                        dq = fmaf(q8[e], ke[e], dq);
+                                        if (kDelta) dk = fmaf(k8[e], ke[e], dk);
+                                    }
+                                }
                             }
-                        }
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            dq0 += __shfl_xor_sync(0xffffffffu, dq0, o);
-                            dq1 += __shfl_xor_sync(0xffffffffu, dq1, o);
-                            if (kDelta) {
-                                dk0 += __shfl_xor_sync(0xffffffffu, dk0, o);
-                                dk1 += __shfl_xor_sync(0xffffffffu, dk1, o);
+                            for (int o = 1; o < 8; o <<= 1) {
+                                dq += __shfl_xor_sync(0xffffffffu, dq, o);
+                                if (kDelta) dk += __shfl_xor_sync(0xffffffffu, dk, o);
                             }
-                        }
-                        if (lane == 0) {
-                            const float w0 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i0]);
-                            sl[oCQ + i0] = w0 * dq0;
-                            if (kDelta) sl[oCK + i0] = w0 * dk0;
-                            if (two) {
-                                const float w1 = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i1]);
-                                sl[oCQ + i1] = w1 * dq1;
-                                if (kDelta) sl[oCK + i1] = w1 * dk1;
+                            if (s8 == 0 && i < len) {
+                                const float w = kVecDecay ? 1.f : expf(lbar_s[0] - L_a[i]);
+                                sl[oCQ + i] = w * dq;
+                                if (kDelta) sl[oCK + i] = w * dk;
                             }
                         }
                     }
+                    float qv[EPL], kv[EPL];
+                    load_vec<float, EPL>(q_s + lane * EPL, qv);
+                    load_vec<float, EPL>(k_s + lane * EPL, kv);
                     if (gwarp == kHalf - 1) {  // q.k for the delta rule, r.(bonus.k) for RWKV6
                         float d = 0.f;
                         float bw[EPL];
