@@ -48,9 +48,10 @@ constexpr int kP64MaxVal = 32;             // (mbarrier storage)
 constexpr int kP64Threads = 32 * (kP64StreamWarps + 4 + 4 + kP64BaseWarps + kP64AuxWarps);  // stream, prep, epilogue, base and aux producers
 constexpr int kP64ScalarWarps = 4;         // prep warps, and as many epilogue warps
 constexpr int kP64BarrierBytes = 2048;
-// hand-over slot (floats): q, k, mul_k, mul_q, lbar, lbar' [6 x 64], ck, cq [2 x 64], scalars [4],
+// hand-over slot (floats): q, k, mul_k, mul_q, lbar, lbar' [6 x 64], ck, cq [2 x kP64MaxCap], scalars [4],
 // the two base-pass results [2][64]
-constexpr int kP64SlotFloats = 6 * 64 + 2 * kMaxCap + 4 + 2 * 64;
+constexpr int kP64MaxCap = 32;             // largest capacity this kernel takes (sizes the coefficient arrays of a slot)
+constexpr int kP64SlotFloats = 6 * 64 + 2 * kP64MaxCap + 4 + 2 * 64;
 constexpr int kP64SlotBytes = (kP64SlotFloats * 4 + 127) / 128 * 128;
 
 // Byte offsets inside a key-side stage and a value-side stage with room for n log entries.
@@ -98,8 +99,8 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
     constexpr bool kPost = OpTraits<OP>::kPostReadout;
     constexpr bool kVecDecay = OpTraits<OP>::kVecDecay;
     constexpr int DL = kVecDecay ? D : 1;
-    constexpr int oQ = 0, oK = 64, oMK = 128, oMQ = 192, oLB = 256, oLN = 320, oCK = 384, oCQ = 384 + kMaxCap,
-                  oSC = 384 + 2 * kMaxCap, oRED = oSC + 4;
+    constexpr int oQ = 0, oK = 64, oMK = 128, oMQ = 192, oLB = 256, oLN = 320, oCK = 384, oCQ = 384 + kP64MaxCap,
+                  oSC = 384 + 2 * kP64MaxCap, oRED = oSC + 4;
 
     constexpr int kEntryBytes = D * (int)(sizeof(IO) + sizeof(UL)) + DL * 4;  // one log entry
     extern __shared__ __align__(128) unsigned char smem[];

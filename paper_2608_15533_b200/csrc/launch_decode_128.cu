@@ -106,7 +106,8 @@ int launch_decode(const StateArgs &st_in, const TokenArgs &tk, cudaStream_t stre
         // one-CTA-per-unit kernel is the faster one (measured on configuration 3's shape at capacity 32:
         // 105 - 144 us per launch against ~80 - 95 us from 17 entries on), so it keeps the larger capacities.
         static const int max_cap = env_int("DELTALOG_P64_MAX_CAP", 16);
-        if (impl != 1 && dev.sms > 0 && fits && st.cap <= max_cap && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
+        if (impl != 1 && dev.sms > 0 && fits && st.cap <= max_cap && st.cap <= kP64MaxCap &&
+            (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
             auto kernel = decode_pipelined_d64_kernel<OP, IO, UL>;
             const int smem = p64_smem_bytes(c64);
             if (int rc = ensure_smem(kernel, smem)) return rc;
