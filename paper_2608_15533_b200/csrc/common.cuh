@@ -275,6 +275,26 @@ __device__ __forceinline__ void rank_update(float4 (&s)[NP], int len, LoadA load
 #endif
 }
 
+// The same update with one scalar FMA per element (identical results: every element sees the same fused
+// multiply-adds in the same order).  Two resident CTAs that stay on an SM for the whole launch share the
+// packed-FMA pipe badly -- the older CTA's warps are served first and the younger one's rank update takes
+// three times as long (measured) -- while scalar FMAs are shared evenly.
+template <int NP, typename LoadA, typename LoadU>
+__device__ __forceinline__ void rank_update_scalar(float4 (&s)[NP], int len, LoadA load_a, LoadU load_u) {
+    static_assert(NP % 4 == 0, "rows come in groups of four");
+    for (int i = 0; i < len; ++i) {
+        const float4 u = load_u(i);
+#pragma unroll
+        for (int p4 = 0; p4 < NP / 4; ++p4) {
+            const float4 a = load_a(i, p4);
+            s[4 * p4 + 0] = fma4(a.x, u, s[4 * p4 + 0]);
+            s[4 * p4 + 1] = fma4(a.y, u, s[4 * p4 + 1]);
+            s[4 * p4 + 2] = fma4(a.z, u, s[4 * p4 + 2]);
+            s[4 * p4 + 3] = fma4(a.w, u, s[4 * p4 + 3]);
+        }
+    }
+}
+
 // Resolve the pool slot of batch row b; returns false when the row must be skipped.
 __device__ __forceinline__ bool resolve_slot(const int32_t *slot_idx, int b, int num_slots, int32_t *status,
                                              int tid, int &slot) {

@@ -7,6 +7,7 @@
 #include <cstdint>
 #include <cstdlib>
 #include <map>
+#include <tuple>
 #include <mutex>
 #include <type_traits>
 #include <utility>
@@ -51,6 +52,31 @@ int ensure_smem(K kernel, size_t bytes) {
     }
     g = bytes;
     return DELTALOG_OK;
+}
+
+// CTAs of a kernel that an SM holds at once with the given shared memory (after ensure_smem), looked up once per
+// (device, kernel, size): the resident kernels size their grids by it.
+template <typename K>
+int resident_ctas(K kernel, int threads, size_t smem) {
+    static std::mutex mu;
+    static std::map<std::tuple<int, const void *, size_t>, int> known;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const auto key = std::make_tuple(dev, reinterpret_cast<const void *>(kernel), smem);
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = known.find(key);
+    if (it != known.end()) return it->second;
+    // Several CTAs of ~100 KB each only fit when the SM's L1 / shared-memory split is at its largest; left to itself the
+    // driver may pick a split that holds one.
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        cudaGetLastError();
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, smem) != cudaSuccess) {
+        cudaGetLastError();
+        n = 0;
+    }
+    known[key] = n;
+    return n;
 }
 
 // Launch with programmatic stream serialisation: the caller promised (DELTALOG_HINT_BASE_UNTOUCHED) that

@@ -1,4 +1,4 @@
-"""The give-up path of the bounded waits inside the persistent decode kernel.
+"""The give-up path of the bounded waits inside the persistent decode kernel and the resident fused-step kernel.
 
 Every wait on an mbarrier in that kernel is bounded in time; when one runs out, the CTA raises its
 abort flag, all roles leave their loops, copies still in flight are waited for (again bounded) and
@@ -59,6 +59,23 @@ CHILD = textwrap.dedent("""
     assert rel_err(np.stack([f64(o).reshape(N, -1) for o in outs]), ref["out"]) <= 2e-2
     assert rel_err(f64(state.S_base).reshape(N, wl.d, wl.d), ref["S"]) <= 1e-4
     print("wait-timeout path ok")
+
+    # 3. the resident fused-merge-step kernel has one bounded wait (for a unit's tile): the tile of one (row, head)
+    # pair is never requested; the launch returns with the TIMEOUT bit alone, and a fresh state afterwards is fine
+    os.environ["DELTALOG_TEST_DROP_ITEM"] = str(296 + 3)            # the second unit of resident CTA 3
+    state = dl.State(desc, S0.clone())
+    t = toks[0]
+    dl.decode_merge_step(desc, state, t["q"], t["k"], t["v"], t["g"], beta=t["beta"])
+    torch.cuda.synchronize()
+    assert int(state.status.item()) == dl.STATUS_TIMEOUT, int(state.status.item())
+    os.environ["DELTALOG_TEST_DROP_ITEM"] = "-1"
+    state = dl.State(desc, S0.clone())
+    outs = [dl.decode_merge_step(desc, state, t["q"], t["k"], t["v"], t["g"], beta=t["beta"]) for t in toks]
+    torch.cuda.synchronize()
+    assert int(state.status.item()) == 0
+    assert rel_err(np.stack([f64(o).reshape(N, -1) for o in outs]), ref["out"]) <= 2e-2
+    assert rel_err(f64(state.S_base).reshape(N, wl.d, wl.d), ref["S"]) <= 1e-4
+    print("fused-step wait-timeout path ok")
 """)
 
 
@@ -66,3 +83,4 @@ def test_a_wait_that_runs_out_ends_the_launch_with_the_timeout_bit_and_leaves_th
     proc = subprocess.run([sys.executable, "-c", CHILD.format(root=str(ROOT))], capture_output=True, text=True, timeout=900)
     assert proc.returncode == 0, proc.stdout[-2000:] + proc.stderr[-3000:]
     assert "wait-timeout path ok" in proc.stdout
+    assert "fused-step wait-timeout path ok" in proc.stdout
