@@ -27,7 +27,7 @@ ROOT = Path(__file__).resolve().parent.parent
 DEFAULT_OUT = ROOT / "profiles" / "dram_traffic.json"
 
 _UNIT = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9, "Tbyte": 1e12}
-FAMILIES = (("decode_merge_step", "fused"), ("decode_pipelined", "decode"), ("decode_append", "decode"),
+FAMILIES = (("fused_step_resident", "fused"), ("decode_merge_step", "fused"), ("decode_pipelined", "decode"), ("decode_append", "decode"),
             ("decode_multi", "decode_multi"), ("merge_tc", "merge"), ("merge_kernel", "merge"),
             ("eager_step", "eager"))
 
