@@ -12,8 +12,9 @@
 // vectors of unit n+1 as soon as unit n has consumed its own (raw key-side rows and token after the
 // weights are formed, value-side rows after the rank update), so every operand of a unit has a
 // unit's compute and store time to arrive and the only wait left is a short one for the tile.
-// Measured per launch against one unit per CTA: configuration 1's shape 114 -> 110 us, configuration
-// 2's 266 -> 222 us, configuration 3's 144 -> 125 us.  (The plain merge, whose CTAs have no readout /
+// Measured per launch against one unit per CTA at capacity 16: configuration 1's shape 114 -> 110-113 us
+// (capacity 8: 101 -> 88 us), configuration 2's 266 -> 222 us, configuration 3's 144 -> 125 us; the launcher
+// uses it up to capacity 16.  (The plain merge, whose CTAs have no readout /
 // reduction chain to hide, does not gain: one unit per CTA already runs at 0.96 of the copy peak
 // there and this scheme was 5-10 % behind it, so the merge keeps merge_kernel.)
 //

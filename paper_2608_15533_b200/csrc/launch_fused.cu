@@ -8,12 +8,15 @@ namespace {
 
 template <int OP, int DK, int DV, typename IO, typename UL, typename BT>
 int launch_fused_step(const StateArgs &st, const TokenArgs &tk, cudaStream_t stream) {
-    // The resident kernel (the next unit's tile, log and token in flight while a unit is computed and stored) where its
-    // shared memory leaves room for the same number of CTAs per SM as one unit per CTA has: up to capacity 16 at head
-    // size 128.  DELTALOG_MAT_PREFETCH=0 keeps one unit per CTA.
+    // The resident kernel (the next unit's tile, log and token in flight while a unit is computed and stored) up to
+    // capacity 16, where its shared memory leaves room for the same number of CTAs per SM as one unit per CTA has.
+    // Its rank update costs more per live entry (scalar FMAs: 3.3 against 1.6 us per entry and launch on configuration
+    // 1's shape), so one unit per CTA is the faster kernel beyond that (measured at capacity 8 / 16 / 24: 88 / 113 /
+    // 140 us against 101 / 114 / 127 us; KDA shape at 16: 223 against 268 us; RWKV6 shape at 16 / 32: 125 / 181 against
+    // 144 / 176 us).  DELTALOG_MAT_PREFETCH=0 keeps one unit per CTA everywhere.
     static const int prefetch = env_int("DELTALOG_MAT_PREFETCH", 1);
     const DeviceInfo &dev = device_info();
-    if (prefetch && dev.sms > 0 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
+    if (prefetch && dev.sms > 0 && st.cap <= 16 && (OpTraits<OP>::kVecDecay || st.cap % 4 == 0)) {
         auto kernel = fused_step_resident_kernel<OP, DK, DV, IO, UL, BT>;
         const size_t bytes = FusedResidentLayout<OP, DK, DV, IO, UL, BT>(st.cap).bytes;
         constexpr int kWant = mat_threads<DK, DV>() <= 128 ? 4 : 2;
