@@ -170,6 +170,58 @@ def test_fused_step_padding_bad_slots_and_slot_indirection():
     assert rel_err(f64(state.S_base), f64(S_e)) <= 1e-5
 
 
+@pytest.mark.parametrize("op,d", [(GDN, 128), (KDA, 128), (RWKV6, 64)])
+def test_fused_step_walk_over_many_units_with_padding_and_indirection(op, d):
+    """A batch large enough that every resident CTA of the fused-step kernel walks over several units, with a
+    permuted slot list, padding rows and one slot outside the pool in the walk: after a few appends, the fused
+    step's outputs and folded states agree with the eager kernel run on a materialised copy of the pool, rows
+    that were skipped are untouched, and their units keep their logs."""
+    import paper_2608_15533_b200 as dl
+
+    batch, H, cap, appends = 150, 8, 8, 3                      # 1200 (row, head) pairs: 2-4 per resident CTA
+    wl = small(op, d, torch.bfloat16, batch=batch, H=H, steps=appends + 1, num_slots=batch + 10)
+    src = workloads.TokenSource(wl, device="cpu")
+    S0 = src.initial_state().to(DEV)
+    bonus = src.bonus().to(DEV) if op == RWKV6 else None
+    desc = make_desc(wl, cap, 1.0)
+    state = dl.State(desc, S0.clone())
+    g = torch.Generator().manual_seed(5)
+    slots = torch.randperm(wl.slots, generator=g)[:batch].to(torch.int32)
+    pad_rows = [3, 77, 78, 149]
+    bad_row = 40
+    slots[pad_rows] = -1
+    slots[bad_row] = wl.slots + 5
+    slot_idx = slots.to(DEV)
+    S_e = S0.clone()                                            # the eager kernel's pool
+    tok = None
+    for t in range(appends + 1):
+        tok = {k_: (v_.to(DEV) if v_ is not None else None) for k_, v_ in src.token().items()}
+        if t < appends:
+            dl.decode_step(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,
+                           slot_idx=slot_idx)
+            dl.eager_step(desc, S_e, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,
+                          slot_idx=slot_idx)
+    torch.cuda.synchronize()
+    state.status.zero_()                                        # (the appends flagged the bad slot as well)
+    out = torch.full((batch, H, d), 3.0, dtype=wl.io_dtype, device=DEV)
+    dl.decode_merge_step(desc, state, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,
+                         slot_idx=slot_idx, out=out)
+    out_e = dl.eager_step(desc, S_e, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"], u_bonus=bonus,
+                          slot_idx=slot_idx)
+    torch.cuda.synchronize()
+    assert int(state.status.item()) == dl.STATUS_BAD_SLOT
+    ran = [b for b in range(batch) if b not in pad_rows and b != bad_row]
+    for b in pad_rows + [bad_row]:
+        assert bool((out[b] == 3.0).all())
+    assert rel_err(f64(out[ran]), f64(out_e[ran])) <= 1.6e-2    # two bf16 roundings of nearly equal fp32 values
+    used = slots[ran].long()
+    assert rel_err(f64(state.S_base[used]), f64(S_e[used])) <= 1e-5
+    assert int(state.log_len[used].abs().max()) == 0            # folded
+    unused = torch.tensor(sorted(set(range(wl.slots)) - set(used.tolist())))
+    assert torch.equal(state.S_base[unused], S0[unused])        # never touched
+    assert int(state.log_len[unused].abs().max()) == 0
+
+
 def test_mixing_fused_steps_and_token_less_merges():
     """The two ways of materialising can be mixed freely on one state."""
     import paper_2608_15533_b200 as dl
