@@ -37,7 +37,9 @@ __global__ void __launch_bounds__(mat_threads<DK, DV>(), mat_threads<DK, DV>() <
     static_assert(NT >= DK && NT >= (kDelta ? 2 : 1) * DV, "one thread per key channel and per output column");
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.x / st.H, h = blockIdx.x % st.H;
+    // (pairs from the last to the first, see merge_kernel: what is written last is what the next decode step reads first)
+    const int pair = gridDim.x - 1 - blockIdx.x;
+    const int b = pair / st.H, h = pair % st.H;
     int slot;
     if (!resolve_slot(tk.slot_idx, b, st.num_slots, st.status, tid, slot)) return;
     const size_t unit = (size_t)slot * st.H + h, row = (size_t)b * st.H + h;

@@ -102,7 +102,7 @@ fused_step_resident_kernel(StateArgs st, TokenArgs tk, int32_t n_pairs, int32_t 
 
     // pair (batch row * H + head) -> unit (slot * H + head), or -1 for a padding row and a slot outside the pool
     auto unit_of = [&](int pair) -> int {
-        if (pair >= n_pairs) return -1;
+        if (pair < 0) return -1;
         int slot;
         if (!resolve_slot(tk.slot_idx, pair / H, st.num_slots, st.status, tid, slot)) return -1;
         return slot * H + pair % H;
@@ -140,7 +140,9 @@ fused_step_resident_kernel(StateArgs st, TokenArgs tk, int32_t n_pairs, int32_t 
         gsc = (!kVecDecay && tk.g) ? tk.g[pair] : 0.f;  // no gate: plain linear attention
     };
 
-    int pair = blockIdx.x;
+    // Pairs are taken from the last to the first: the tiles written last (still in L2 when the kernel ends) are
+    // then the ones the next decode step, which walks upwards from pair 0, reads first.
+    int pair = n_pairs - 1 - (int)blockIdx.x;
     int unit = unit_of(pair);
     int len = 0;
     float beta = 0.f, gsc = 0.f;
@@ -155,8 +157,8 @@ fused_step_resident_kernel(StateArgs st, TokenArgs tk, int32_t n_pairs, int32_t 
     const int c4 = tid % C4, rl = tid / C4;
     uint32_t phase = 0;
     bool timed_out = false;
-    for (; pair < n_pairs; pair += gridDim.x) {
-        const int npair = pair + gridDim.x;
+    for (; pair >= 0; pair -= gridDim.x) {
+        const int npair = pair - (int)gridDim.x;
         const int nunit = unit_of(npair);
         float bonus_r[EPL];
 #pragma unroll

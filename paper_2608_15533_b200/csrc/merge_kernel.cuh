@@ -73,7 +73,9 @@ merge_kernel(StateArgs st, const int32_t *slot_idx, int32_t only_if_full, int32_
         unit = (size_t)s_unit[cand];
         if (cand > 0) __syncthreads();  // the previous candidate's shared-memory operands are no longer read
     } else {
-        const int pair = blockIdx.x;
+        // CTAs take the pairs from the last to the first: the tiles written last (and still in L2 when the
+        // kernel ends) are then the ones the next decode step, which walks upwards from pair 0, reads first
+        const int pair = gridDim.x - 1 - blockIdx.x;
         int slot;
         if (!resolve_slot(slot_idx, pair / st.H, st.num_slots, st.status, tid, slot)) return;
         unit = (size_t)slot * st.H + pair % st.H;

@@ -62,7 +62,7 @@ CHILD = textwrap.dedent("""
 
     # 3. the resident fused-merge-step kernel has one bounded wait (for a unit's tile): the tile of one (row, head)
     # pair is never requested; the launch returns with the TIMEOUT bit alone, and a fresh state afterwards is fine
-    os.environ["DELTALOG_TEST_DROP_ITEM"] = str(296 + 3)            # the second unit of resident CTA 3
+    os.environ["DELTALOG_TEST_DROP_ITEM"] = str(296 + 3)            # one (row, head) pair of the 320
     state = dl.State(desc, S0.clone())
     t = toks[0]
     dl.decode_merge_step(desc, state, t["q"], t["k"], t["v"], t["g"], beta=t["beta"])
