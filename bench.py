@@ -26,6 +26,7 @@ ranks.
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import math
 import os
@@ -184,6 +185,10 @@ class Rig:
                                     ulog_dtype=io if ulog16 else None,
                                     hints=dl.HINT_BASE_UNTOUCHED | dl.HINT_SLOTS_STABLE, base_dtype=base)
         self.chain = os.environ.get("DELTALOG_BENCH_CHAIN", "1") != "0"
+        # Consecutive decode steps of a state walk over the batch in alternating directions (an ordering hint, same
+        # results): a step then starts with the base tiles the step before read last, which are still in L2.
+        self.alternate = os.environ.get("DELTALOG_BENCH_ALTERNATE", "1") != "0"
+        self._descs = {}
         self.states, self.rings, self.bonus = [], [], []
         for layer in range(layers):
             src = workloads.TokenSource(wl, device=device, seed=wl.seed + 1000 * seed_offset + layer)
@@ -206,10 +211,22 @@ class Rig:
             # delay == t mod cap hold a full log; their slots, listed per residue, are what the merge gets
             self.full_slots = [self.slot_idx[self.delay == r].contiguous() for r in range(cap)]
 
-    def decode(self, t, layer=0, slot_idx=None, chained=False):
-        """``chained``: the launch in front of this one on the stream was a decode step of this state."""
+    def desc_for(self, chained=False, down=False):
+        """The descriptor with the hints of one decode call: ``chained`` = the launch in front of it on the stream
+        was a decode step of this state; ``down`` = walk over the batch from the last unit to the first."""
+        hints = (self.desc_chained.hints if (chained and self.chain) else 0) | \
+                (self.dl.HINT_WALK_DOWN if (down and self.alternate) else 0)
+        if hints not in self._descs:
+            self._descs[hints] = dataclasses.replace(self.desc, hints=hints)
+        return self._descs[hints]
+
+    def decode(self, t, layer=0, slot_idx=None, chained=False, fill=None):
+        """``chained``: the launch in front of this one on the stream was a decode step of this state.  ``fill``: the
+        step's place in its cycle (default t mod cap): odd places walk downwards -- the merge and the fused step walk
+        downwards themselves, so place 0 walks upwards."""
         tok = self.rings[layer][t % self.RING]
-        self.dl.decode_step(self.desc_chained if (chained and self.chain) else self.desc, self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
+        place = (t % self.cap) if fill is None else fill
+        self.dl.decode_step(self.desc_for(chained, down=bool(place & 1)), self.states[layer], tok["q"], tok["k"], tok["v"], tok["g"],
                             beta=tok["beta"], u_bonus=self.bonus[layer],
                             slot_idx=self.slot_idx if slot_idx is None else slot_idx, out=self.out)
 
@@ -554,7 +571,7 @@ def time_paper_cycle(rig: Rig, steps: int):
         elif t % M == M - 1:
             dl.decode_merge_step(*args, slot_idx=rig.slot_idx, **kw)
         else:   # every append but the first after the fused step follows a decode step of this state
-            desc = rig.desc_chained if (rig.chain and rig.layers == 1 and t % M != 0) else rig.desc
+            desc = rig.desc_for(chained=(rig.layers == 1 and t % M != 0), down=bool((t % M) & 1))
             dl.decode_step(desc, *args[1:], slot_idx=rig.slot_idx, **kw)
 
     stream = torch.cuda.Stream(device=rig.device)

@@ -6,7 +6,7 @@
 """
 from . import traffic  # noqa: F401
 from .binding import (  # noqa: F401
-    BF16, F32, GDN, GLA, HINT_BASE_UNTOUCHED, HINT_SLOTS_STABLE, KDA, LINATTN, RETNET, RWKV6, STATUS_BAD_SLOT, STATUS_LOG_FULL, STATUS_TIMEOUT, DeltalogError, Desc,
+    BF16, F32, GDN, GLA, HINT_BASE_UNTOUCHED, HINT_SLOTS_STABLE, HINT_WALK_DOWN, KDA, LINATTN, RETNET, RWKV6, STATUS_BAD_SLOT, STATUS_LOG_FULL, STATUS_TIMEOUT, DeltalogError, Desc,
     HostLane, HostStaging, State, decode_merge_step, decode_step, decode_steps, decode_step_host_overlapped, decode_step_host, decode_step_host_static, eager_step, build_id, launch_count, load_library, merge, packed_host_tokens, reset_slots,
     status_string, version,
 )

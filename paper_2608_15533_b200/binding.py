@@ -15,7 +15,7 @@ from typing import Optional
 import torch
 
 GDN, KDA, RWKV6, LINATTN, RETNET, GLA = 0, 1, 2, 3, 4, 5
-HINT_BASE_UNTOUCHED, HINT_SLOTS_STABLE = 1, 2
+HINT_BASE_UNTOUCHED, HINT_SLOTS_STABLE, HINT_WALK_DOWN = 1, 2, 4
 _DELTA_RULE = (GDN, KDA)            # b = beta (v - S'^T k): U log in fp32
 _VEC_DECAY = (KDA, RWKV6, GLA)      # one log-decay per key channel
 F32, BF16 = 0, 1

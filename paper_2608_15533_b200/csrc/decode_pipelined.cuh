@@ -275,8 +275,12 @@ decode_pipelined_kernel(StateArgs st, TokenArgs tk, PipeCfg cfg) {
 
     const int total = tk.B * st.H;
     const bool slots_early = tk.slot_idx == nullptr || (tk.hints & DELTALOG_HINT_SLOTS_STABLE) != 0;
-    const int first = blockIdx.x, stride = gridDim.x;
-    const int n_items = (total - first + stride - 1) / stride;
+    // A CTA takes the units blockIdx.x, blockIdx.x + gridDim.x, ... -- counted from the last unit downwards under
+    // DELTALOG_HINT_WALK_DOWN (unit = first + i * stride either way).
+    const int n_items = (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const bool walk_down = (tk.hints & DELTALOG_HINT_WALK_DOWN) != 0;
+    const int first = walk_down ? total - 1 - (int)blockIdx.x : (int)blockIdx.x;
+    const int stride = walk_down ? -(int)gridDim.x : (int)gridDim.x;
     const int cap = st.cap, H = st.H;
 
     // ---- the aux ring is laid out for the longest LIVE log among this CTA's units ----------------------

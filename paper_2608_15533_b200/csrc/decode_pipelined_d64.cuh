@@ -151,8 +151,11 @@ __global__ void __launch_bounds__(kP64Threads, 1) decode_pipelined_d64_kernel(St
 
     const int total = tk.B * st.H;
     const bool slots_early = tk.slot_idx == nullptr || (tk.hints & DELTALOG_HINT_SLOTS_STABLE) != 0;
-    const int first = blockIdx.x, stride = gridDim.x;
-    const int n_items = first < total ? (total - first + stride - 1) / stride : 0;
+    // units blockIdx.x, blockIdx.x + gridDim.x, ... -- counted from the last unit downwards under DELTALOG_HINT_WALK_DOWN
+    const int n_items = (int)blockIdx.x < total ? (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const bool walk_down = (tk.hints & DELTALOG_HINT_WALK_DOWN) != 0;
+    const int first = walk_down ? total - 1 - (int)blockIdx.x : (int)blockIdx.x;
+    const int stride = walk_down ? -(int)gridDim.x : (int)gridDim.x;
     const int cap = st.cap, H = st.H;
     auto slot_of = [&](int i) { return reinterpret_cast<float *>(slots + (size_t)(i % NS) * kP64SlotBytes); };
     constexpr int kFirstBaseWarp = kP64StreamWarps + 2 * kP64ScalarWarps;
