@@ -701,7 +701,8 @@ def time_eager_loop(rig: Rig, S: torch.Tensor, steps: int, use_graph: bool = Tru
     def launch_steps(n):
         for t in range(n):
             tok = rig.rings[0][t % rig.RING]
-            dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+            # (the comparator gets the same courtesy as the decode steps: alternating walking directions)
+            dl.eager_step(rig.desc_for(down=bool(t & 1)), S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
                           u_bonus=rig.bonus[0], out=rig.out)
 
     steps = max(steps // rig.RING, 2) * rig.RING

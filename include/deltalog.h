@@ -123,7 +123,9 @@ typedef struct {
  *       A caller that sets the bit on every other step of a state lets each step begin with the base
  *       tiles the step before read last, which are still in L2 (configuration 1: -1.7 % per step).
  *       deltalog_merge and deltalog_decode_merge_step walk downwards by themselves, so the step after
- *       one of them should walk upwards.  Kernels with one CTA per unit ignore the bit.
+ *       one of them should walk upwards.  deltalog_eager_step honours the bit as well (its CTAs are
+ *       numbered downwards: a step then begins with the tiles the step before wrote last); the other
+ *       kernels with one CTA per unit ignore it.
  */
 enum { DELTALOG_HINT_BASE_UNTOUCHED = 1, DELTALOG_HINT_SLOTS_STABLE = 2, DELTALOG_HINT_WALK_DOWN = 4 };
 

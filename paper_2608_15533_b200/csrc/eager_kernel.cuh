@@ -21,7 +21,10 @@ eager_step_kernel(void *S, int32_t num_slots, int32_t H, float scale, int32_t *s
     constexpr int C4 = DV / 4, RL = kThreads / C4, NP = DK / RL, EPL = DK / 32;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int b = blockIdx.x / H, h = blockIdx.x % H;
+    // (DELTALOG_HINT_WALK_DOWN: CTAs take the units from the last to the first -- alternated from step to step, a
+    // step begins with the tiles the step before wrote last, which are still in L2)
+    const int pair = (tk.hints & DELTALOG_HINT_WALK_DOWN) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
+    const int b = pair / H, h = pair % H;
     int slot;
     if (!resolve_slot(tk.slot_idx, b, num_slots, status, tid, slot)) return;
     const size_t unit = (size_t)slot * H + h, row = (size_t)b * H + h;

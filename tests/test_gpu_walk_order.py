@@ -61,3 +61,26 @@ def test_walking_downwards_changes_no_bit(op, d, batch, H):
         assert torch.equal(st.S_base, S0), name                  # a decode step never writes the base
     live = slots[slots >= 0].long()
     assert int(ref.log_len[live].min()) == steps and int(ref.log_len.sum()) == steps * live.numel() * H
+
+
+@pytest.mark.parametrize("op,d", [(GDN, 128), (RWKV6, 64)])
+def test_eager_step_walking_downwards_changes_no_bit(op, d):
+    import paper_2608_15533_b200 as dl
+
+    batch, H = 24, 8
+    wl = Workload(f"walk_eager_op{op}", op, batch, H, d, 4, (1,), io_dtype=torch.bfloat16)
+    src = workloads.TokenSource(wl, device="cpu")
+    S0 = src.initial_state().to(DEV)
+    bonus = src.bonus().to(DEV) if op == RWKV6 else None
+    toks = [{k: (v.to(DEV) if v is not None else None) for k, v in src.token().items()} for _ in range(4)]
+    base = make_desc(wl, 1, 1.0)
+    res = []
+    for pattern in (lambda t: 0, lambda t: dl.HINT_WALK_DOWN if t & 1 else 0):
+        S, outs = S0.clone(), []
+        for t, tok in enumerate(toks):
+            outs.append(dl.eager_step(dataclasses.replace(base, hints=pattern(t)), S, tok["q"], tok["k"], tok["v"], tok["g"],
+                                      beta=tok["beta"], u_bonus=bonus))
+        torch.cuda.synchronize()
+        res.append((torch.stack(outs), S))
+    assert torch.equal(res[0][0].view(torch.int16), res[1][0].view(torch.int16))
+    assert torch.equal(res[0][1], res[1][1])
