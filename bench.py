@@ -912,7 +912,7 @@ def hot_loop_for_profilers(rig: Rig, args):
         S = rig.states[0].S_base
         for t in range(args.steps):
             tok = rig.rings[0][t % rig.RING]
-            rig.dl.eager_step(rig.desc, S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
+            rig.dl.eager_step(rig.desc_for(down=bool(t & 1)), S, tok["q"], tok["k"], tok["v"], tok["g"], beta=tok["beta"],
                               u_bonus=rig.bonus[0], out=rig.out)
     else:   # the paper's cycle: cap appends, then the fused merge step
         M = rig.cap + 1
