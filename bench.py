@@ -934,6 +934,9 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the capacity sweep, eager and CPU legs")
     ap.add_argument("--state", default="fp32", choices=["fp32", "bf16"],
                     help="dtype of the dense state; bf16 is the 16-bit-state variant (the configurations name fp32)")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="with --only-hot-loop: run this many layers of a multi-layer configuration instead of all "
+                         "(a profiler capture of the serving shape that holds a few GB instead of 29)")
     ap.add_argument("--only-hot-loop", action="store_true",
                     help="warm-up and then --steps steps as plain launches, nothing else (for profiler captures)")
     ap.add_argument("--hot-loop-kind", default="cycle", choices=["cycle", "eager", "paper"],
@@ -955,6 +958,9 @@ def main():
     cap, K = args.cap, args.steps
     warmup = max(args.warmup, 3)
     layers = wl.layers
+    if args.layers:
+        assert args.only_hot_loop and 1 <= args.layers <= wl.layers, "--layers goes with --only-hot-loop"
+        layers = args.layers
     base16 = args.state == "bf16"
     # weak scaling: the global batch is `size` times the configuration's rows, sharded by rows
     first_row, n_rows = launch.shard_rows(size * wl.batch, size, rank)
